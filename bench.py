@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the HPSGD replica-update + merge path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+A "step" is one round of the whole path on one workload: one local step of every one of
+the K simulated workers followed by one synchronisation (merge).  The metric is
+parameter updates per second, K*P*steps / time.  One JSON line is printed by rank 0.
+
+  * own arm (default): inputs resident in HBM, timed on the device with CUDA events;
+    plus `e2e` (host gradient buffers through hpsgd_local_step_host, host copy of the
+    global model every step), `roofline` for the kernels and `cpu_baseline`.
+  * --impl reference: the CPU oracle, as it stands, on a bounded sample of the workload.
+
+With N > 1 (torchrun) every rank runs an independent replica of the same workload (the
+path has no inter-GPU exchange); time is the max over ranks, value the sum of units.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "parameter_updates_per_sec"
+UNIT = "K*P elems/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------ helpers
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def local_bytes_per_elem(cfg):
+    """Algorithmic HBM bytes per parameter and worker of one local step."""
+    g = 2 if cfg.grad_dtype == "bf16" else 4
+    return g + 8 + (8 if cfg.momentum else 0)
+
+
+def merge_bytes_per_index(cfg):
+    """Algorithmic HBM bytes per parameter index of one merge: (2K + 4) * 4."""
+    return (2 * cfg.K + 4) * 4
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ CPU oracle legs
+def oracle_sample_run(cfg, seconds, sample_params=4_000_000, min_rounds=2, max_rounds=None):
+    """Time the CPU oracle on the first `sample_params` parameters of the workload.
+
+    Gradient generation is outside the timed part (as on the GPU).  Returns
+    (elems_per_s, rounds, seconds_timed, description)."""
+    from oracle.ref import RefHPSGD
+    P = min(cfg.P, sample_params)
+    idx = np.arange(P, dtype=np.int64)
+    o = RefHPSGD(P, cfg.K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+    o.set_global(cfg.initial_global(idx))
+    grads = [[cfg.stored_gradient(i, t, idx) for i in range(cfg.K)] for t in range(2)]
+    rounds, spent = 0, 0.0
+    while True:
+        g = grads[rounds % 2]
+        t0 = time.perf_counter()
+        for i in range(cfg.K):
+            o.local_step(i, g[i])
+        o.sync_merge()
+        spent += time.perf_counter() - t0
+        rounds += 1
+        if max_rounds is not None and rounds >= max_rounds:
+            break
+        if max_rounds is None and rounds >= min_rounds and spent >= seconds:
+            break
+    o.close()
+    desc = ("first %d of %d parameters of %s, all K=%d workers, %d rounds (local steps + merge; "
+            "sparse rows given as dense zeros), single thread" % (P, cfg.P, cfg.name, cfg.K, rounds))
+    return cfg.K * P * rounds / spent, rounds, spent, desc, P
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle, one bounded sample per step."""
+    for _ in range(max(0, args.warmup)):
+        oracle_sample_run(cfg, 0, sample_params=args.ref_sample, max_rounds=1)
+    t_total, units = 0.0, 0
+    desc = ""
+    for _ in range(args.steps):
+        eps, rounds, spent, desc, P = oracle_sample_run(cfg, 0, sample_params=args.ref_sample, max_rounds=1)
+        t_total += spent
+        units += cfg.K * P
+    value = units / t_total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic (counter-hash gradients)",
+        "config": workload_config(cfg, {"sample": "each step = one round on the first %d parameters" % min(cfg.P, args.ref_sample)}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(cfg, extra=None):
+    c = {"workload": "%s: %s" % (cfg.name, cfg.note), "K": cfg.K, "P": cfg.P, "tensors": len(cfg.sizes),
+         "lr": cfg.lr, "momentum": cfg.momentum, "weight_decay": cfg.weight_decay,
+         "grad_dtype": cfg.grad_dtype, "staleness": cfg.staleness, "local_steps_per_merge": 1}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ------------------------------------------------------------------------------ distributed plumbing
+def dist_setup(n_gpus):
+    """Returns (rank, world, local_rank, dist-module-or-None)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world <= 1:
+        return 0, 1, 0, None
+    import torch.distributed as dist
+    backend = os.environ.get("HPSGD_BENCH_BACKEND", "nccl")
+    dist.init_process_group(backend=backend)
+    return dist.get_rank(), dist.get_world_size(), int(os.environ.get("LOCAL_RANK", "0")), dist
+
+
+def aggregate(dist, device, elapsed_ms, units):
+    """Whole-job figures: time = max over ranks, units = sum over ranks."""
+    if dist is None:
+        return elapsed_ms, units
+    import torch
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def run_gpu(args, cfg):
+    import torch
+    import paper_2009_02701_b200 as hp
+
+    rank, world, local_rank, dist = dist_setup(args.gpus)
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    lay = cfg.layout
+    K, P, P_pad = cfg.K, cfg.P, lay.P_pad
+    bf16 = cfg.grad_dtype == "bf16"
+    gdt = torch.int16 if bf16 else torch.float32
+    gsz = 2 if bf16 else 4
+    kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
+
+    # ---- state: arena and streams come from torch, the library only computes
+    hp.hpsgd_destroy()
+    if len(cfg.sizes) > 1:
+        hp.hpsgd_set_layout(list(cfg.sizes))
+    nbytes = hp.hpsgd_arena_bytes(P_pad, K, hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0,
+                                  cfg.sparse[1] if cfg.sparse else 0)
+    arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
+    base = arena.data_ptr() + (-arena.data_ptr()) % 256
+    main, side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    hp.hpsgd_bind(base, nbytes, main, side)
+    hp.hpsgd_init(P, K, cfg.lr, cfg.momentum, cfg.seed)
+    if cfg.weight_decay:
+        hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, cfg.weight_decay)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, args.chunks)
+    if cfg.sparse:
+        hp.hpsgd_set_sparse_segment(*cfg.sparse)
+
+    # ---- inputs: `nbuf` rounds of gradients for all K workers, generated on the device
+    nbuf = args.grad_buffers
+    grads = torch.empty((nbuf, K, P_pad), dtype=gdt, device=dev)
+    sparse_in = None
+    if cfg.sparse:
+        rows_max = cfg.sparse[1]
+        cols = cfg.sparse[2]
+        sparse_in = []
+        for b in range(nbuf):
+            per_worker = []
+            for i in range(K):
+                idx = torch.from_numpy(cfg.sparse_rows(i, b)).to(dev)
+                vals = torch.empty(idx.numel() * cols, dtype=gdt, device=dev)
+                hp.hpsgd_gen_row_vals(vals, i, b, kind, cfg.grad_scale, idx, idx.numel())
+                per_worker.append((idx, vals))
+            sparse_in.append(per_worker)
+    for b in range(nbuf):
+        for i in range(K):
+            hp.hpsgd_gen_grads(grads[b, i], i, b, kind, cfg.grad_scale)
+    hp.hpsgd_synchronize()
+
+    def one_round(t):
+        b = t % nbuf
+        if cfg.sparse:
+            descs = [hp.make_desc(grads[b, i], sparse_in[b][i][0], sparse_in[b][i][0].numel(), sparse_in[b][i][1])
+                     for i in range(K)]
+            if args.per_worker:
+                for i in range(K):
+                    hp.hpsgd_local_step_ex(i, descs[i])
+            else:
+                hp.hpsgd_local_step_all_ex(descs)
+        elif args.per_worker:
+            for i in range(K):
+                hp.hpsgd_local_step(i, grads[b, i])
+        else:
+            hp.hpsgd_local_step_all(grads[b], P_pad * gsz)
+        hp.hpsgd_sync_merge()
+
+    # ---- warm-up, then the timed region
+    for t in range(args.warmup):
+        one_round(t)
+    hp.hpsgd_synchronize()
+    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)
+    hp.hpsgd_profile_read()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = hp.hpsgd_launch_count()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record(main)
+    for t in range(args.steps):
+        one_round(args.warmup + t)
+    main.wait_stream(side)
+    end.record(main)
+    torch.cuda.synchronize(dev)
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    elapsed_ms = start.elapsed_time(end)
+    launches = hp.hpsgd_launch_count() - launches0
+    local_ms, local_n, merge_ms, merge_n = hp.hpsgd_profile_read()
+    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 0)
+    units = K * P * args.steps
+    job_ms, job_units = aggregate(dist, dev, elapsed_ms, units)
+    value = job_units / (job_ms * 1e-3)
+
+    # ---- roofline of the two kernels from the event pairs recorded inside the timed region
+    peak, peak_src = measured_peak()
+    merge_launch_bytes = merge_bytes_per_index(cfg) * P * args.steps / max(merge_n, 1)
+    local_launch_bytes = local_bytes_per_elem(cfg) * P * K * args.steps / max(local_n, 1)
+    merge_gbs = merge_bytes_per_index(cfg) * P * args.steps / (merge_ms * 1e-3) / 1e9 if merge_ms else 0.0
+    local_gbs = local_bytes_per_elem(cfg) * P * K * args.steps / (local_ms * 1e-3) / 1e9 if local_ms else 0.0
+    kernels = {
+        "merge_kernel": {"launches": merge_n, "avg_ms": merge_ms / max(merge_n, 1), "algorithmic_bytes_per_launch": merge_launch_bytes,
+                         "achieved": merge_gbs, "frac": merge_gbs / peak, "frac_of_nominal_8TBs": merge_gbs / NOMINAL_HBM_GBS},
+        "local_step_kernel": {"launches": local_n, "avg_ms": local_ms / max(local_n, 1), "algorithmic_bytes_per_launch": local_launch_bytes,
+                              "achieved": local_gbs, "frac": local_gbs / peak, "frac_of_nominal_8TBs": local_gbs / NOMINAL_HBM_GBS},
+    }
+    dominant = "local_step_kernel" if local_ms >= merge_ms else "merge_kernel"
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved"], "peak": peak,
+                "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": None,
+                "peak_source": peak_src, "nominal_peak": NOMINAL_HBM_GBS, "kernels": kernels,
+                "note": "event pairs around each launch on its own stream inside the timed region; "
+                        "with chunks > 1 the two kernels overlap and share HBM"}
+    round_bytes = (local_bytes_per_elem(cfg) * K + merge_bytes_per_index(cfg)) * P
+    roofline["round_achieved"] = round_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
+    roofline["round_frac"] = roofline["round_achieved"] / peak
+
+    # ---- end to end: host gradient buffers in, host copy of the global model out, every step
+    e2e = None
+    if rank == 0 or dist is not None:
+        e2e = run_e2e(args, cfg, hp, torch, dev, grads, dist)
+
+    line = None
+    if rank == 0:
+        cpu = None
+        if args.cpu_seconds > 0:
+            eps, rounds, spent, desc, _ = oracle_sample_run(cfg, args.cpu_seconds)
+            cpu = {"value": eps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+                   "seconds": spent}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": job_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic (counter-hash gradients generated on the device, %d rounds cycled)" % nbuf,
+            "config": workload_config(cfg, {
+                "schedule": {"overlap": args.overlap, "chunks": args.chunks,
+                             "local_step_call": "per worker" if args.per_worker else "all K in one call"},
+                "l2": "inputs larger than L2 (state + gradients are tens of GB)",
+                "multi_gpu": "independent replicas, no inter-GPU exchange"}),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+    hp.hpsgd_destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+
+
+def run_e2e(args, cfg, hp, torch, dev, grads, dist):
+    """Same metric with host buffers: every step copies each worker's gradient from pinned
+    host memory (hpsgd_local_step_host) and reads the global model back (hpsgd_copy_global)."""
+    K, P, P_pad = cfg.K, cfg.P, cfg.layout.P_pad
+    gsz = 2 if cfg.grad_dtype == "bf16" else 4
+    if cfg.sparse:
+        hp.hpsgd_set_sparse_segment(-1, 0, 0)      # host path: dense gradients with zero rows
+    nhost = min(K, args.e2e_host_buffers)
+    host = [torch.empty(P_pad, dtype=grads.dtype).pin_memory() for _ in range(nhost)]
+    for j in range(nhost):
+        host[j].copy_(grads[0, j])
+    out = torch.empty(P, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize(dev)
+
+    def one_step():
+        for i in range(K):
+            hp.hpsgd_local_step_host(i, host[i % nhost])
+        hp.hpsgd_sync_merge()
+        hp.hpsgd_copy_global(out)
+
+    for _ in range(args.e2e_warmup):
+        one_step()
+    hp.hpsgd_synchronize()
+    if dist is not None:
+        dist.barrier()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    start.record()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        one_step()
+    end.record()
+    torch.cuda.synchronize(dev)
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    ms = max(start.elapsed_time(end), wall_ms)     # the device-to-host copy blocks the host
+    job_ms, job_units = aggregate(dist, dev, ms, K * P * args.e2e_steps)
+    if cfg.sparse:
+        hp.hpsgd_set_sparse_segment(*cfg.sparse)
+    return {"value": job_units / (job_ms * 1e-3), "unit": UNIT, "ms_per_step": job_ms / args.e2e_steps,
+            "steps": args.e2e_steps, "h2d_bytes_per_step": K * P_pad * gsz, "d2h_bytes_per_step": P * 4,
+            "host_buffers": "%d pinned gradient buffers cycled over the K workers" % nhost}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=workloads.names())
+    ap.add_argument("--overlap", type=int, default=1)
+    ap.add_argument("--chunks", type=int, default=1)
+    ap.add_argument("--per-worker", action="store_true", help="K hpsgd_local_step calls instead of one batched call")
+    ap.add_argument("--grad-buffers", type=int, default=2, help="rounds of device-resident gradients to cycle")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-warmup", type=int, default=1)
+    ap.add_argument("--e2e-host-buffers", type=int, default=4)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU oracle baseline budget (0 = skip)")
+    ap.add_argument("--ref-sample", type=int, default=4_000_000, help="parameters per step of --impl reference")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
+    cfg = workloads.get(args.workload)
+
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return 0
+        run_reference(args, cfg)
+        return 0
+    run_gpu(args, cfg)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,286 @@
+/*
+ * libhpsgd: the HPSGD replica update and delayed merge on one NVIDIA B200 (sm_100a).
+ *
+ * K simulated workers each hold a flat fp32 replica r_i of a P-parameter model.  A local
+ * step applies one worker's gradient to its replica (Algorithm 2 of the HPSGD paper); a
+ * synchronisation averages the K replica changes in the fixed order i = 0..K-1 (the
+ * AllReduce of Algorithm 3, mean as in Eq. 1), commits the average obtained at the
+ * PREVIOUS synchronisation to the global model w (Algorithm 3, first step; Section 3.2,
+ * last paragraph: the global update lags its all-reduce by one synchronisation) and
+ * re-clones every replica from the updated w (Algorithm 2, "make replica").
+ *
+ * Conventions
+ *   - All pointers are DEVICE pointers unless the name or comment says "host".
+ *   - Every entry point returns HPSGD_OK (0) or a negative hpsgd_status; nothing throws,
+ *     aborts or exits across this boundary.  hpsgd_last_error() gives the text of the
+ *     last failure.  Argument errors are detected before any GPU work is issued.
+ *   - The library is a process-wide singleton (the four core calls carry no handle) and is
+ *     not thread-safe: call it from one host thread.
+ *   - hpsgd_local_step* and hpsgd_sync_merge only ENQUEUE work.  An asynchronous CUDA
+ *     failure is reported by the next call as HPSGD_E_CUDA.
+ *   - Flat layout: tensor t of the parameter set starts at a multiple of 32 elements
+ *     (128 bytes) inside every flat buffer; the gaps ("pads") hold zero, must receive
+ *     zero gradient, and are not parameters.  P_pad is the padded length.  With a single
+ *     tensor P_pad = P rounded up to 32.
+ *   - There is no CPU fallback: without a CUDA device every call that needs one fails
+ *     with HPSGD_E_CUDA.
+ */
+#ifndef HPSGD_H_
+#define HPSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum hpsgd_status {
+    HPSGD_OK = 0,
+    HPSGD_E_BADARG = -1,      /* invalid argument; nothing was enqueued */
+    HPSGD_E_STATE = -2,       /* call not legal in the current state (e.g. before hpsgd_init) */
+    HPSGD_E_NOMEM = -3,       /* arena too small or device allocation failed */
+    HPSGD_E_CUDA = -4,        /* a CUDA call failed; see hpsgd_last_error() */
+    HPSGD_E_TIMEOUT = -5,     /* a bounded device-side wait gave up */
+    HPSGD_E_UNSUPPORTED = -6  /* size beyond a documented limit */
+} hpsgd_status;
+
+/* Keys of hpsgd_set_option. */
+enum {
+    HPSGD_OPT_WEIGHT_DECAY = 1, /* lambda >= 0, coupled L2 at the replica: gd = g + lambda*r. Default 0. */
+    HPSGD_OPT_STALENESS = 2,    /* 1 (default): commit the previous average, the paper's schedule.
+                                   0: commit the fresh average at once (Eq. 2 / Local SGD). */
+    HPSGD_OPT_GRAD_DTYPE = 3,   /* HPSGD_F32 (default) or HPSGD_BF16: storage type of gradients. */
+    HPSGD_OPT_OVERLAP = 4,      /* 1 (default): merge on the side stream, ordered against local
+                                   steps by events; 0: everything on the main stream. */
+    HPSGD_OPT_CHUNKS = 5,       /* number of index ranges the schedule is cut into (1..1024).
+                                   Results do not depend on it. Default 1. */
+    HPSGD_OPT_PROFILE = 6       /* 1: bracket every local-step call and every merge with CUDA
+                                   events on the stream it runs on (see hpsgd_profile_read). */
+};
+
+enum { HPSGD_F32 = 0, HPSGD_BF16 = 1 };
+
+/* Kinds of synthetic gradient (hpsgd_gen_grads). */
+enum { HPSGD_GEN_UNIFORM = 0, HPSGD_GEN_GAUSS = 1 };
+
+/* Flags of hpsgd_arena_bytes. */
+enum { HPSGD_ARENA_MOMENTUM = 1 };
+
+/* ------------------------------------------------------------------------------------
+ * The four core calls.
+ * ---------------------------------------------------------------------------------- */
+
+/*
+ * Create the state for K workers and P parameters: global model w, pending averaged
+ * change D = 0, replicas r_i = w and (momentum != 0 only) momentum buffers m_i = 0.
+ * w is filled with seeded uniform values in [-0.1, 0.1) (counter hash, stream 2; see
+ * hpsgd_gen_grads for the hash).  lr is the paper's mu (Algorithm 2 initialisation:
+ * mu >= 0); momentum is the heavy-ball factor beta in [0, 1) (0 = the paper's plain SGD).
+ * If hpsgd_set_layout was called, P must equal the sum of its sizes; otherwise the
+ * parameter set is one tensor of P elements.  If hpsgd_bind supplied an arena it is
+ * used (and must be large enough, else HPSGD_E_NOMEM); otherwise the library allocates
+ * one with cudaMalloc and frees it in hpsgd_destroy.  A second hpsgd_init without
+ * hpsgd_destroy returns HPSGD_E_STATE.  Blocks until the fill has completed.
+ */
+int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed);
+
+/*
+ * One local step of worker `worker` (Algorithm 2, "update replica"; momentum and weight
+ * decay are extensions the paper does not have), element-wise over the flat buffer:
+ *     gd = g + lambda*r_i ;  m_i = beta*m_i + gd ;  r_i = r_i - mu*m_i
+ * each line one fused multiply-add in binary32, round to nearest even.  `grads` is a
+ * device buffer of P_pad elements in the flat layout, fp32 or bf16 per
+ * HPSGD_OPT_GRAD_DTYPE, 16-byte aligned, zero in the pads.  It is borrowed: keep it
+ * valid and unchanged until the work has run (hpsgd_synchronize, or a stream wait on
+ * the main stream).  Several local steps per worker between two merges are legal
+ * (Section 3.2: several local trainings per synchronisation); a worker with none
+ * contributes a zero change.  Enqueued on the main stream.
+ */
+int hpsgd_local_step(int worker, const void* grads);
+
+/*
+ * One synchronisation (Algorithm 3 + the replica clone of Algorithm 2), per index j:
+ *     acc  = (r_0 - w) + (r_1 - w) + ... + (r_{K-1} - w)      left to right
+ *     Dnew = acc / (float)K                                    correctly rounded
+ *     staleness 1: w = w + D if this is not the first merge ; D = Dnew
+ *     staleness 0: w = w + Dnew ; D = Dnew
+ *     r_i  = w  for every i
+ * in one fused kernel.  m_i is not touched.  Enqueued on the side stream (main stream
+ * when HPSGD_OPT_OVERLAP is 0) behind all local steps issued so far; later local steps
+ * wait, per index range, for the part of the merge they depend on.
+ */
+int hpsgd_sync_merge(void);
+
+/*
+ * Wait for all enqueued work and return the device pointer to w (P_pad floats, flat
+ * layout, library-owned, valid until hpsgd_destroy).  The pending change D is NOT
+ * flushed into it: after T merges w holds the changes of rounds 0..T-2 (one-
+ * synchronisation delay).  Returns NULL on error.
+ */
+const float* hpsgd_get_global(void);
+
+/* ------------------------------------------------------------------------------------
+ * Layout, memory and streams (all optional; call before hpsgd_init).
+ * ---------------------------------------------------------------------------------- */
+
+/*
+ * Padded length for a list of tensor sizes (host array); if offsets_out (host, n_tensors
+ * entries) is not NULL it receives each tensor's start in the flat buffers.  Pure
+ * function, no GPU needed.  Returns a negative hpsgd_status on bad input.
+ */
+int64_t hpsgd_layout_padded(int n_tensors, const int64_t* sizes, int64_t* offsets_out);
+
+/* Declare the tensor sizes (host array, each > 0) used by the next hpsgd_init. */
+int hpsgd_set_layout(int n_tensors, const int64_t* sizes);
+
+/*
+ * Bytes of device memory the state needs: w, D, K replicas, K momentum buffers when
+ * flags has HPSGD_ARENA_MOMENTUM, plus the row->slot scratch map for a sparse-row
+ * tensor of up to `sparse_rows` rows per worker (0 if unused) and a small table.
+ */
+size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows);
+
+/*
+ * Lend device memory and streams for the next hpsgd_init.  `arena` (256-byte aligned,
+ * `bytes` long) stays owned by the caller and must outlive hpsgd_destroy; pass NULL / 0
+ * to let the library allocate.  main_stream / side_stream are cudaStream_t handles
+ * owned by the caller (e.g. torch streams); pass NULL to let the library create its own.
+ */
+int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream);
+
+/* Set an option (keys above).  Legal after hpsgd_init, between rounds. */
+int hpsgd_set_option(int key, double value);
+
+/* ------------------------------------------------------------------------------------
+ * Batched and sparse-row local steps.
+ * ---------------------------------------------------------------------------------- */
+
+/*
+ * Gradient of one worker with one tensor given as sparse rows.  `dense` is as in
+ * hpsgd_local_step; inside the span of the sparse tensor its contents are ignored.
+ * The sparse tensor (declared by hpsgd_set_sparse_segment) is [rows x cols]; row_idx
+ * (device, int32, ascending, unique, each in [0, rows)) lists the n_rows rows that carry
+ * a gradient and row_vals (device, [n_rows x cols], same dtype as dense, 16-byte
+ * aligned) their values.  Rows not listed have gradient ZERO and are still stepped
+ * (momentum decays and moves the replica, weight decay applies): the result equals
+ * a dense step with zero rows.  row_idx == NULL or n_rows == 0 means no sparse tensor
+ * rows are active.  Unsorted, duplicate or out-of-range rows are the caller's error.
+ */
+typedef struct hpsgd_grad_desc {
+    const void* dense;
+    const int32_t* row_idx;
+    int32_t n_rows;
+    const void* row_vals;
+} hpsgd_grad_desc;
+
+/* Declare tensor `tensor_id` as the [rows x cols] sparse-row tensor (cols % 8 == 0,
+ * rows*cols == its size).  tensor_id < 0 removes the declaration.  After hpsgd_init.
+ * The row->slot scratch map lives in the arena; a caller-supplied arena must have been
+ * sized with sparse_rows >= rows, else HPSGD_E_NOMEM. */
+int hpsgd_set_sparse_segment(int tensor_id, int64_t rows, int64_t cols);
+
+/* hpsgd_local_step with a sparse-row tensor (desc is a host struct, read during the call). */
+int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc);
+
+/*
+ * One local step of ALL K workers in one launch per index range: worker i reads its
+ * dense gradient at (char*)grads + i * worker_stride_bytes (16-byte aligned stride).
+ * Same arithmetic as K calls of hpsgd_local_step; the launches are issued range by
+ * range so that, with HPSGD_OPT_CHUNKS > 1, the merge of a range can start while later
+ * ranges are still being stepped.
+ */
+int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes);
+
+/* The same for K sparse-row descriptors (host array of K structs).  K <= 32. */
+int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs);
+
+/* ------------------------------------------------------------------------------------
+ * Host-buffer convenience (end-to-end use) and inspection.
+ * ---------------------------------------------------------------------------------- */
+
+/*
+ * hpsgd_local_step with `host_grads` in HOST memory (P_pad elements, flat layout;
+ * pinned memory gives asynchronous copies).  The library copies it to an internal
+ * double-buffered staging area (allocated with cudaMalloc on first use, freed in
+ * hpsgd_destroy) and enqueues the step; the host buffer may be reused once the call
+ * returns only if it is NOT pinned; for pinned memory keep it unchanged until
+ * hpsgd_synchronize.
+ */
+int hpsgd_local_step_host(int worker, const void* host_grads);
+
+/* Overwrite w from a HOST array of the P parameters (un-padded concatenation of the
+ * tensors) and reset D = 0, r_i = w, m_i = 0, merge count 0.  Blocking. */
+int hpsgd_set_global_host(const float* host_w, int64_t n);
+
+/* Wait for all work, then copy the P parameters of w (un-padded concatenation) to a
+ * HOST array of n = P floats.  Blocking. */
+int hpsgd_copy_global(float* host_out, int64_t n);
+
+/* Device pointers (P_pad floats each) to worker's replica and momentum buffer (*m = NULL
+ * when momentum == 0), and to the pending change D.  Any out pointer may be NULL.
+ * Does not synchronise. */
+int hpsgd_get_replica(int worker, const float** r, const float** m);
+int hpsgd_get_pending(const float** D);
+
+/* Current sizes: any out pointer may be NULL. */
+int hpsgd_get_sizes(int64_t* P, int64_t* P_pad, int* K, int64_t* merges);
+
+/* Start of tensor t in the flat buffers, or a negative hpsgd_status. */
+int64_t hpsgd_tensor_offset(int tensor_id);
+
+/* ------------------------------------------------------------------------------------
+ * Synthetic gradients generated on the device (inputs for benchmarks and large tests).
+ * ---------------------------------------------------------------------------------- */
+
+/*
+ * Fill `out` (device, P_pad elements of the current HPSGD_OPT_GRAD_DTYPE, flat layout,
+ * pads zero) with the gradient of (worker, step) from the counter hash seeded by
+ * hpsgd_init's seed:
+ *   mix(x): x ^= x>>32; x *= M1; x ^= x>>29; x *= M2; x ^= x>>32         (uint64)
+ *   key = mix(seed + M3);  ctr = stream<<60 | step<<40 | worker<<32 | idx
+ *   h = mix(mix(ctr ^ key) + M4);  u24 = h>>40;  v24 = (h>>16) & 0xFFFFFF
+ *   M1..M4 = frac(sqrt 2, 3, 5, 7) * 2^64 with the low bit set
+ * with idx the index in the UN-padded concatenation of the tensors (< 2^32), stream 0.
+ *   HPSGD_GEN_UNIFORM: g = (float)scale * ((int)u24 - 2^23) * 2^-23
+ *   HPSGD_GEN_GAUSS:   g = (float)(scale * sqrt(-2 ln((u24+1) 2^-24)) * cos(2 pi v24 2^-24)), in binary64
+ * bf16 storage rounds that fp32 value to nearest even.  If a sparse-row tensor is
+ * declared, its rows whose mask hash (stream 1, idx = row) has u24 >= 1677721 are zero.
+ * Enqueued on the main stream.  step < 2^20, worker < 256.
+ */
+int hpsgd_gen_grads(void* out, int worker, int step, int kind, double scale);
+
+/* Values of the listed rows of the sparse-row tensor, [n_rows x cols] into `out`, same
+ * generator and dtype as hpsgd_gen_grads.  Enqueued on the main stream. */
+int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
+                       const int32_t* row_idx, int32_t n_rows);
+
+/* ------------------------------------------------------------------------------------
+ * Housekeeping.
+ * ---------------------------------------------------------------------------------- */
+
+/* Wait for all enqueued work on both streams. */
+int hpsgd_synchronize(void);
+
+/*
+ * With HPSGD_OPT_PROFILE on: total device milliseconds and number of kernel launches of
+ * the local-step kernels and of the merge kernels since the last read, measured with
+ * CUDA event pairs recorded around each launch on the stream it ran on.  Synchronises
+ * and resets the totals.  Any out pointer may be NULL.
+ */
+int hpsgd_profile_read(double* local_ms, int64_t* local_launches,
+                       double* merge_ms, int64_t* merge_launches);
+
+/* Number of kernels this library has launched since hpsgd_init. */
+int64_t hpsgd_launch_count(void);
+
+/* Text of the last error (static storage, never NULL). */
+const char* hpsgd_last_error(void);
+
+/* Free everything the library allocated; the state can be created again afterwards. */
+int hpsgd_destroy(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HPSGD_H_ */

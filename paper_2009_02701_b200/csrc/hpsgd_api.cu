@@ -1,0 +1,887 @@
+// C ABI of libhpsgd: state, validation, stream/event schedule and kernel launches.
+// The contract of every entry point is documented in include/hpsgd.h.
+#include "../../include/hpsgd.h"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "hpsgd_kernels.cuh"
+
+namespace {
+
+using namespace hpsgd;
+
+constexpr int64_t kAlignElems = 32;        // tensor starts: multiples of 32 elements
+constexpr int64_t kRowAlignElems = 64;     // rows of r / m: multiples of 256 bytes
+constexpr size_t kAlignBytes = 256;        // arena regions
+constexpr int kMaxChunks = 1024;
+constexpr int kMaxTensors = 4096;
+constexpr int64_t kChunkGrainVec = 2048;   // chunk boundaries: multiples of 8192 elements
+
+char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                      \
+    do {                                                                                    \
+        cudaError_t e_ = (expr);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return fail(HPSGD_E_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));      \
+    } while (0)
+
+#define TRY(expr)                \
+    do {                         \
+        int rc_ = (expr);        \
+        if (rc_) return rc_;     \
+    } while (0)
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct EventPair {
+    cudaEvent_t a, b;
+    int kind;       // 0 local step, 1 merge
+};
+
+struct Pending {                // configuration collected before hpsgd_init
+    std::vector<int64_t> sizes;
+    void* arena = nullptr;
+    size_t arena_bytes = 0;
+    cudaStream_t main = nullptr, side = nullptr;
+    bool have_streams = false;
+} g_pending;
+
+struct Ctx {
+    bool inited = false;
+    int64_t P = 0, P_pad = 0, stride = 0;  // stride: floats between consecutive workers' rows
+    int K = 0;
+    float lr = 0.f, beta = 0.f, lambda = 0.f;
+    uint64_t seed = 0, key = 0;
+    int staleness = 1, grad_dtype = HPSGD_F32, overlap = 1, chunks = 1, profile = 0;
+    std::vector<int64_t> sizes, offsets, starts;
+    int64_t* d_table = nullptr;            // offsets | starts | sizes, on the device
+    char* arena = nullptr;
+    size_t arena_bytes = 0;
+    bool own_arena = false;
+    float *w = nullptr, *D = nullptr, *r = nullptr, *m = nullptr;
+    int32_t* slot = nullptr;               // [K][slot_cap] row -> slot scratch map
+    int64_t slot_cap = 0;
+    bool own_slot = false;
+    cudaStream_t main = nullptr, side = nullptr, copy = nullptr;
+    bool own_streams = false;
+    std::vector<cudaEvent_t> ev_local, ev_merge;
+    std::vector<char> local_recorded, merge_unwaited;
+    bool D_valid = false;
+    int64_t merges = 0;
+    int64_t launches = 0;
+    int sm_count = 148;
+    int sp_tensor = -1;                    // sparse-row tensor
+    int64_t sp_rows = 0, sp_cols = 0;
+    void* stage[2] = {nullptr, nullptr};   // staging of hpsgd_local_step_host
+    cudaEvent_t stage_copied[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
+    bool stage_used[2] = {false, false};
+    int stage_next = 0;
+    std::vector<EventPair> prof;           // profiling
+    double prof_ms[2] = {0, 0};
+    int64_t prof_launches[2] = {0, 0};
+} g;
+
+int check_async()
+{
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) return fail(HPSGD_E_CUDA, "CUDA error: %s", cudaGetErrorString(e));
+    return HPSGD_OK;
+}
+
+int64_t layout_of(const std::vector<int64_t>& sizes, std::vector<int64_t>* offsets, std::vector<int64_t>* starts)
+{
+    int64_t pos = 0, flat = 0;
+    for (int64_t s : sizes) {
+        if (offsets) offsets->push_back(pos);
+        if (starts) starts->push_back(flat);
+        pos += (s + kAlignElems - 1) / kAlignElems * kAlignElems;
+        flat += s;
+    }
+    return pos;
+}
+
+// Regions of the arena, in order: w | D | r[K] | m[K] | table | slot maps (the rest).
+struct ArenaPlan {
+    size_t w, D, r, m, table, slot, fixed;
+};
+
+ArenaPlan plan_arena(int64_t stride, int K, bool momentum)
+{
+    ArenaPlan a{};
+    const size_t row = (size_t)stride * 4;
+    size_t pos = 0;
+    a.w = pos; pos += row;
+    a.D = pos; pos += row;
+    a.r = pos; pos += row * K;
+    a.m = pos; if (momentum) pos += row * K;
+    a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kAlignBytes);
+    a.slot = pos;
+    a.fixed = pos;
+    return a;
+}
+
+// Index range [v_lo, v_hi), in 4-element vectors, of schedule chunk c.
+void chunk_range(int c, int64_t* v_lo, int64_t* v_hi)
+{
+    const int64_t nvec = g.P_pad / 4;
+    const int64_t grains = (nvec + kChunkGrainVec - 1) / kChunkGrainVec;
+    auto edge = [&](int k) { return std::min(nvec, grains * k / g.chunks * kChunkGrainVec); };
+    *v_lo = edge(c);
+    *v_hi = (c == g.chunks - 1) ? nvec : edge(c + 1);
+}
+
+// Grid: enough blocks to cover `items` at `per_block` each, capped at one full wave of
+// resident blocks (SM count x blocks the kernel can keep resident per SM).
+template <typename Kern>
+int grid_for(Kern kern, int64_t items, int64_t per_block)
+{
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0) != cudaSuccess || occ < 1) occ = 1;
+    const int64_t need = std::max<int64_t>(1, (items + per_block - 1) / per_block);
+    return (int)std::min<int64_t>(need, (int64_t)g.sm_count * occ);
+}
+
+// ---------------------------------------------------------------------------- profiling
+int prof_begin(cudaStream_t s, int kind, EventPair* ep)
+{
+    if (!g.profile) return HPSGD_OK;
+    ep->kind = kind;
+    CUDA_TRY(cudaEventCreate(&ep->a));
+    CUDA_TRY(cudaEventCreate(&ep->b));
+    CUDA_TRY(cudaEventRecord(ep->a, s));
+    return HPSGD_OK;
+}
+
+int prof_end(cudaStream_t s, EventPair* ep)
+{
+    if (!g.profile) return HPSGD_OK;
+    CUDA_TRY(cudaEventRecord(ep->b, s));
+    g.prof.push_back(*ep);
+    return HPSGD_OK;
+}
+
+int prof_resolve()
+{
+    for (EventPair& ep : g.prof) {
+        CUDA_TRY(cudaEventSynchronize(ep.b));
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, ep.a, ep.b));
+        g.prof_ms[ep.kind] += ms;
+        g.prof_launches[ep.kind] += 1;
+        cudaEventDestroy(ep.a);
+        cudaEventDestroy(ep.b);
+    }
+    g.prof.clear();
+    return HPSGD_OK;
+}
+
+// ---------------------------------------------------------------------------- local step
+struct LocalLaunch {
+    int w0, nw;
+    BatchPtrs gp;
+    SparseSeg seg;
+    int64_t v0, nvec;
+    StepParams p;
+};
+
+template <bool BF16, bool MOM, bool WD, bool SPARSE>
+void launch_local(const LocalLaunch& L)
+{
+    constexpr int U = 4;
+    auto kern = local_step_kernel<BF16, MOM, WD, SPARSE, U>;
+    dim3 grid(grid_for(kern, L.nvec, (int64_t)kThreads * U), L.nw);
+    kern<<<grid, kThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.v0, L.nvec, L.p);
+}
+
+template <bool BF16, bool MOM, bool WD>
+void launch_local_s(bool sparse, const LocalLaunch& L)
+{
+    if (sparse) launch_local<BF16, MOM, WD, true>(L);
+    else launch_local<BF16, MOM, WD, false>(L);
+}
+
+template <bool BF16>
+void launch_local_d(bool mom, bool wd, bool sparse, const LocalLaunch& L)
+{
+    if (mom && wd) launch_local_s<BF16, true, true>(sparse, L);
+    else if (mom) launch_local_s<BF16, true, false>(sparse, L);
+    else if (wd) launch_local_s<BF16, false, true>(sparse, L);
+    else launch_local_s<BF16, false, false>(sparse, L);
+}
+
+// Enqueue the local step of workers [w0, w0 + nw) on the main stream, chunk by chunk.
+int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
+{
+    LocalLaunch L{};
+    L.w0 = w0; L.nw = nw; L.gp = gp;
+    L.p = StepParams{-g.lr, g.beta, g.lambda};
+    L.seg = SparseSeg{0, 0, 1};
+    if (sparse) {
+        L.seg.v_begin = g.offsets[g.sp_tensor] / 4;
+        L.seg.v_end = L.seg.v_begin + g.sp_rows * g.sp_cols / 4;
+        L.seg.cols4 = (int32_t)(g.sp_cols / 4);
+    }
+    const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
+    for (int c = 0; c < g.chunks; ++c) {
+        int64_t lo, hi;
+        chunk_range(c, &lo, &hi);
+        if (hi <= lo) continue;
+        if (g.merge_unwaited[c]) {
+            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
+            g.merge_unwaited[c] = 0;
+        }
+        L.v0 = lo; L.nvec = hi - lo;
+        EventPair ep{};
+        TRY(prof_begin(g.main, 0, &ep));
+        if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
+        else launch_local_d<false>(mom, wd, sparse, L);
+        ++g.launches;
+        TRY(prof_end(g.main, &ep));
+        if (g.overlap) {
+            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
+            g.local_recorded[c] = 1;
+        }
+    }
+    return check_async();
+}
+
+// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors.
+int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* gp)
+{
+    for (int i = 0; i < nw; ++i) {
+        int32_t* slot = g.slot + (int64_t)(w0 + i) * g.slot_cap;
+        CUDA_TRY(cudaMemsetAsync(slot, 0xFF, (size_t)g.sp_rows * 4, g.main));     // every row: no slot (-1)
+        const hpsgd_grad_desc& d = descs[i];
+        if (d.row_idx && d.n_rows > 0) {
+            scatter_slots_kernel<<<(d.n_rows + 255) / 256, 256, 0, g.main>>>(slot, d.row_idx, d.n_rows, g.sp_rows);
+            ++g.launches;
+        }
+        gp->slot[i] = slot;
+        gp->row_vals[i] = d.row_vals;
+        gp->dense[i] = d.dense;
+    }
+    return HPSGD_OK;
+}
+
+int check_grad_ptr(const void* p, const char* what)
+{
+    if (!p) return fail(HPSGD_E_BADARG, "%s is NULL", what);
+    if (reinterpret_cast<uintptr_t>(p) % 16) return fail(HPSGD_E_BADARG, "%s is not 16-byte aligned", what);
+    return HPSGD_OK;
+}
+
+int check_desc(const hpsgd_grad_desc* d)
+{
+    if (!d) return fail(HPSGD_E_BADARG, "descriptor is NULL");
+    TRY(check_grad_ptr(d->dense, "dense gradient"));
+    if (d->n_rows < 0 || d->n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows %d out of range", d->n_rows);
+    if (d->n_rows > 0 && d->row_idx) TRY(check_grad_ptr(d->row_vals, "row_vals"));
+    return HPSGD_OK;
+}
+
+int need_init()
+{
+    if (!g.inited) return fail(HPSGD_E_STATE, "hpsgd_init has not been called");
+    return HPSGD_OK;
+}
+
+int check_worker(int worker)
+{
+    if (worker < 0 || worker >= g.K) return fail(HPSGD_E_BADARG, "worker %d outside [0, %d)", worker, g.K);
+    return HPSGD_OK;
+}
+
+int sync_all()
+{
+    CUDA_TRY(cudaStreamSynchronize(g.main));
+    CUDA_TRY(cudaStreamSynchronize(g.side));
+    if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
+    return HPSGD_OK;
+}
+
+int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; blocking
+{
+    const size_t row = (size_t)g.stride * 4;
+    CUDA_TRY(cudaMemsetAsync(g.D, 0, row, g.main));
+    if (g.m) CUDA_TRY(cudaMemsetAsync(g.m, 0, row * g.K, g.main));
+    const int64_t nvec = g.P_pad / 4;
+    clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
+    ++g.launches;
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(g.main));
+    g.D_valid = false;
+    g.merges = 0;
+    std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
+    std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
+    return HPSGD_OK;
+}
+
+int make_chunk_events(int chunks)
+{
+    for (cudaEvent_t e : g.ev_local) cudaEventDestroy(e);
+    for (cudaEvent_t e : g.ev_merge) cudaEventDestroy(e);
+    g.ev_local.assign(chunks, nullptr);
+    g.ev_merge.assign(chunks, nullptr);
+    g.local_recorded.assign(chunks, 0);
+    g.merge_unwaited.assign(chunks, 0);
+    g.chunks = chunks;
+    for (int c = 0; c < chunks; ++c) {
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_local[c], cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_merge[c], cudaEventDisableTiming));
+    }
+    return HPSGD_OK;
+}
+
+GenParams gen_params(int worker, int step, int kind, double scale)
+{
+    GenParams gp{};
+    gp.key = g.key;
+    gp.step = (uint64_t)step;
+    gp.worker = (uint64_t)worker;
+    gp.kind = kind;
+    gp.scale_f = (float)scale;
+    gp.scale_d = scale;
+    if (g.sp_tensor >= 0) {
+        gp.sp_start = g.starts[g.sp_tensor];
+        gp.sp_rows = g.sp_rows;
+        gp.sp_cols = g.sp_cols;
+    }
+    return gp;
+}
+
+int check_gen_args(const void* out, int worker, int step, int kind)
+{
+    TRY(need_init());
+    TRY(check_grad_ptr(out, "output buffer"));
+    if (worker < 0 || worker >= 256) return fail(HPSGD_E_BADARG, "worker must be in [0, 256)");
+    if (step < 0 || step >= (1 << 20)) return fail(HPSGD_E_BADARG, "step must be in [0, 2^20)");
+    if (kind != HPSGD_GEN_UNIFORM && kind != HPSGD_GEN_GAUSS) return fail(HPSGD_E_BADARG, "unknown generator kind");
+    return HPSGD_OK;
+}
+
+void release_all()
+{
+    if (g.main) cudaStreamSynchronize(g.main);
+    if (g.side) cudaStreamSynchronize(g.side);
+    if (g.copy) cudaStreamSynchronize(g.copy);
+    for (EventPair& ep : g.prof) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+    for (cudaEvent_t e : g.ev_local) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : g.ev_merge) if (e) cudaEventDestroy(e);
+    for (int b = 0; b < 2; ++b) {
+        if (g.stage[b]) cudaFree(g.stage[b]);
+        if (g.stage_copied[b]) cudaEventDestroy(g.stage_copied[b]);
+        if (g.stage_free[b]) cudaEventDestroy(g.stage_free[b]);
+    }
+    if (g.copy) cudaStreamDestroy(g.copy);
+    if (g.own_streams) {
+        if (g.main) cudaStreamDestroy(g.main);
+        if (g.side) cudaStreamDestroy(g.side);
+    }
+    if (g.own_slot && g.slot) cudaFree(g.slot);
+    if (g.own_arena && g.arena) cudaFree(g.arena);
+    cudaGetLastError();
+    g = Ctx();
+}
+
+template <int KT>
+void launch_merge(cudaStream_t s, int64_t v0, int64_t nvec, int flags)
+{
+    auto kern = merge_kernel<KT>;
+    kern<<<grid_for(kern, nvec, kThreads), kThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, v0, nvec, flags);
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+const char* hpsgd_last_error(void) { return g_err; }
+
+int64_t hpsgd_layout_padded(int n_tensors, const int64_t* sizes, int64_t* offsets_out)
+{
+    if (n_tensors <= 0 || !sizes) return fail(HPSGD_E_BADARG, "layout: need at least one tensor size");
+    if (n_tensors > kMaxTensors) return fail(HPSGD_E_UNSUPPORTED, "layout: at most %d tensors", kMaxTensors);
+    std::vector<int64_t> s(sizes, sizes + n_tensors), off;
+    for (int64_t x : s)
+        if (x <= 0) return fail(HPSGD_E_BADARG, "layout: tensor sizes must be positive");
+    const int64_t pad = layout_of(s, &off, nullptr);
+    if (offsets_out) std::memcpy(offsets_out, off.data(), sizeof(int64_t) * n_tensors);
+    return pad;
+}
+
+int hpsgd_set_layout(int n_tensors, const int64_t* sizes)
+{
+    if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_set_layout must precede hpsgd_init");
+    const int64_t pad = hpsgd_layout_padded(n_tensors, sizes, nullptr);
+    if (pad < 0) return (int)pad;
+    g_pending.sizes.assign(sizes, sizes + n_tensors);
+    return HPSGD_OK;
+}
+
+size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows)
+{
+    if (P_pad <= 0 || K <= 0 || sparse_rows < 0) return 0;
+    const int64_t stride = (P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
+    const int64_t cap = (sparse_rows + 63) / 64 * 64;
+    return plan_arena(stride, K, (flags & HPSGD_ARENA_MOMENTUM) != 0).fixed + (size_t)cap * 4 * K;
+}
+
+int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream)
+{
+    if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_bind must precede hpsgd_init");
+    if (arena && reinterpret_cast<uintptr_t>(arena) % kAlignBytes)
+        return fail(HPSGD_E_BADARG, "arena must be 256-byte aligned");
+    if ((arena == nullptr) != (bytes == 0))
+        return fail(HPSGD_E_BADARG, "arena and bytes must both be given or both be zero");
+    if ((main_stream == nullptr) != (side_stream == nullptr))
+        return fail(HPSGD_E_BADARG, "give both streams or neither");
+    if (main_stream && main_stream == side_stream)
+        return fail(HPSGD_E_BADARG, "main and side stream must differ");
+    g_pending.arena = arena;
+    g_pending.arena_bytes = bytes;
+    g_pending.main = static_cast<cudaStream_t>(main_stream);
+    g_pending.side = static_cast<cudaStream_t>(side_stream);
+    g_pending.have_streams = main_stream != nullptr;
+    return HPSGD_OK;
+}
+
+int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
+{
+    if (g.inited) return fail(HPSGD_E_STATE, "already initialised; call hpsgd_destroy first");
+    if (P <= 0) return fail(HPSGD_E_BADARG, "P must be positive");
+    if (P >= (int64_t)1 << 32) return fail(HPSGD_E_UNSUPPORTED, "P must be below 2^32");
+    if (K <= 0 || K > 256) return fail(HPSGD_E_BADARG, "K must be in [1, 256]");
+    if (!(lr >= 0.f)) return fail(HPSGD_E_BADARG, "lr must be >= 0");
+    if (!(momentum >= 0.f && momentum < 1.f)) return fail(HPSGD_E_BADARG, "momentum must be in [0, 1)");
+    std::vector<int64_t> sizes = g_pending.sizes;
+    if (sizes.empty()) sizes.push_back(P);
+    int64_t sum = 0;
+    for (int64_t s : sizes) sum += s;
+    if (sum != P)
+        return fail(HPSGD_E_BADARG, "P = %lld does not match the layout total %lld", (long long)P, (long long)sum);
+
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10)
+        return fail(HPSGD_E_CUDA, "built for sm_100a only; device is sm_%d%d", prop.major, prop.minor);
+
+    g = Ctx();
+    g.sm_count = prop.multiProcessorCount;
+    g.P = P; g.K = K; g.lr = lr; g.beta = momentum; g.seed = seed;
+    g.key = mix64(seed + kM3);
+    g.sizes = sizes;
+    g.P_pad = layout_of(sizes, &g.offsets, &g.starts);
+    g.stride = (g.P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
+    const bool mom = momentum != 0.f;
+    const ArenaPlan a = plan_arena(g.stride, K, mom);
+
+    if (g_pending.arena) {
+        if (g_pending.arena_bytes < a.fixed) {
+            g = Ctx();
+            return fail(HPSGD_E_NOMEM, "arena of %zu bytes is smaller than the %zu needed", g_pending.arena_bytes, a.fixed);
+        }
+        g.arena = static_cast<char*>(g_pending.arena);
+        g.arena_bytes = g_pending.arena_bytes;
+        g.slot_cap = (int64_t)((g.arena_bytes - a.fixed) / ((size_t)4 * K)) / 64 * 64;
+        g.slot = g.slot_cap ? reinterpret_cast<int32_t*>(g.arena + a.slot) : nullptr;
+    } else {
+        void* p = nullptr;
+        cudaError_t e = cudaMalloc(&p, a.fixed);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            g = Ctx();
+            return fail(HPSGD_E_NOMEM, "cudaMalloc of %zu bytes failed: %s", a.fixed, cudaGetErrorString(e));
+        }
+        g.arena = static_cast<char*>(p);
+        g.arena_bytes = a.fixed;
+        g.own_arena = true;
+    }
+    g.w = reinterpret_cast<float*>(g.arena + a.w);
+    g.D = reinterpret_cast<float*>(g.arena + a.D);
+    g.r = reinterpret_cast<float*>(g.arena + a.r);
+    g.m = mom ? reinterpret_cast<float*>(g.arena + a.m) : nullptr;
+    g.d_table = reinterpret_cast<int64_t*>(g.arena + a.table);
+
+    if (g_pending.have_streams) {
+        g.main = g_pending.main;
+        g.side = g_pending.side;
+    } else {
+        g.own_streams = true;
+        if (cudaStreamCreateWithFlags(&g.main, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&g.side, cudaStreamNonBlocking) != cudaSuccess) {
+            release_all();
+            return fail(HPSGD_E_CUDA, "could not create streams");
+        }
+    }
+    g.inited = true;
+    int rc = make_chunk_events(1);
+    if (rc) { release_all(); return rc; }
+
+    // device table: offsets | starts | sizes
+    const size_t n = sizes.size();
+    std::vector<int64_t> table(3 * n);
+    for (size_t t = 0; t < n; ++t) {
+        table[t] = g.offsets[t];
+        table[n + t] = g.starts[t];
+        table[2 * n + t] = sizes[t];
+    }
+    cudaError_t e = cudaMemcpyAsync(g.d_table, table.data(), table.size() * 8, cudaMemcpyHostToDevice, g.main);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(g.main);
+    if (e == cudaSuccess) e = cudaMemsetAsync(g.w, 0, (size_t)g.stride * 4, g.main);
+    if (e != cudaSuccess) {
+        release_all();
+        return fail(HPSGD_E_CUDA, "state set-up failed: %s", cudaGetErrorString(e));
+    }
+    GenParams gp = gen_params(0, 0, 2, 0.0);
+    gen_flat_kernel<false><<<grid_for(gen_flat_kernel<false>, g.P_pad, kThreads), kThreads, 0, g.main>>>(
+        g.w, g.P_pad, g.d_table, g.d_table + n, g.d_table + 2 * n, (int)n, gp);
+    ++g.launches;
+    rc = reset_state_from_w();
+    if (rc) { release_all(); return rc; }
+    g_pending = Pending();
+    return HPSGD_OK;
+}
+
+int hpsgd_destroy(void)
+{
+    release_all();
+    g_pending = Pending();
+    return HPSGD_OK;
+}
+
+int hpsgd_synchronize(void)
+{
+    TRY(need_init());
+    TRY(sync_all());
+    return check_async();
+}
+
+int hpsgd_set_option(int key, double value)
+{
+    TRY(need_init());
+    switch (key) {
+    case HPSGD_OPT_WEIGHT_DECAY:
+        if (!(value >= 0.0)) return fail(HPSGD_E_BADARG, "weight decay must be >= 0");
+        g.lambda = (float)value;
+        return HPSGD_OK;
+    case HPSGD_OPT_STALENESS:
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "staleness must be 0 or 1");
+        if (g.merges) return fail(HPSGD_E_STATE, "staleness can only change before the first merge");
+        g.staleness = (int)value;
+        return HPSGD_OK;
+    case HPSGD_OPT_GRAD_DTYPE:
+        if (value != HPSGD_F32 && value != HPSGD_BF16) return fail(HPSGD_E_BADARG, "unknown gradient dtype");
+        g.grad_dtype = (int)value;
+        return HPSGD_OK;
+    case HPSGD_OPT_OVERLAP:
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "overlap must be 0 or 1");
+        TRY(sync_all());                   // the schedule may only change while idle
+        g.overlap = (int)value;
+        std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
+        std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
+        return HPSGD_OK;
+    case HPSGD_OPT_CHUNKS:
+        if (!(value >= 1.0 && value <= kMaxChunks && value == (double)(int)value))
+            return fail(HPSGD_E_BADARG, "chunks must be an integer in [1, %d]", kMaxChunks);
+        TRY(sync_all());
+        return make_chunk_events((int)value);
+    case HPSGD_OPT_PROFILE:
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "profile must be 0 or 1");
+        TRY(prof_resolve());
+        g.profile = (int)value;
+        return HPSGD_OK;
+    default:
+        return fail(HPSGD_E_BADARG, "unknown option %d", key);
+    }
+}
+
+int hpsgd_set_sparse_segment(int tensor_id, int64_t rows, int64_t cols)
+{
+    TRY(need_init());
+    if (tensor_id < 0) {
+        g.sp_tensor = -1;
+        g.sp_rows = g.sp_cols = 0;
+        return HPSGD_OK;
+    }
+    if (tensor_id >= (int)g.sizes.size()) return fail(HPSGD_E_BADARG, "tensor %d does not exist", tensor_id);
+    if (rows <= 0 || cols <= 0 || cols % 8)
+        return fail(HPSGD_E_BADARG, "rows must be positive and cols a positive multiple of 8");
+    if (rows > INT32_MAX) return fail(HPSGD_E_UNSUPPORTED, "too many rows");
+    if (rows * cols != g.sizes[tensor_id]) return fail(HPSGD_E_BADARG, "rows*cols does not match the tensor size");
+    if (rows > g.slot_cap) {
+        if (!g.own_arena)
+            return fail(HPSGD_E_NOMEM, "arena has room for %lld sparse rows per worker, %lld needed",
+                        (long long)g.slot_cap, (long long)rows);
+        // library-owned memory: the map is its own allocation, kept until hpsgd_destroy
+        TRY(sync_all());
+        if (g.own_slot && g.slot) cudaFree(g.slot);
+        g.slot = nullptr; g.slot_cap = 0; g.own_slot = false;
+        const int64_t cap = (rows + 63) / 64 * 64;
+        void* p = nullptr;
+        cudaError_t e = cudaMalloc(&p, (size_t)cap * 4 * g.K);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(HPSGD_E_NOMEM, "cudaMalloc of the slot map failed: %s", cudaGetErrorString(e));
+        }
+        g.slot = static_cast<int32_t*>(p);
+        g.slot_cap = cap;
+        g.own_slot = true;
+    }
+    g.sp_tensor = tensor_id;
+    g.sp_rows = rows;
+    g.sp_cols = cols;
+    return HPSGD_OK;
+}
+
+// ------------------------------------------------------------------------- local steps
+int hpsgd_local_step(int worker, const void* grads)
+{
+    TRY(need_init());
+    TRY(check_worker(worker));
+    TRY(check_grad_ptr(grads, "grads"));
+    BatchPtrs gp{};
+    gp.dense[0] = grads;
+    return enqueue_local(worker, 1, gp, false);
+}
+
+int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc)
+{
+    TRY(need_init());
+    TRY(check_worker(worker));
+    if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
+    TRY(check_desc(desc));
+    BatchPtrs gp{};
+    TRY(enqueue_slot_maps(worker, 1, desc, &gp));
+    return enqueue_local(worker, 1, gp, true);
+}
+
+int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes)
+{
+    TRY(need_init());
+    TRY(check_grad_ptr(grads, "grads"));
+    const int64_t esz = g.grad_dtype == HPSGD_BF16 ? 2 : 4;
+    if (worker_stride_bytes % 16 || worker_stride_bytes < g.P_pad * esz)
+        return fail(HPSGD_E_BADARG, "worker stride must be a multiple of 16 bytes and cover P_pad elements");
+    for (int w0 = 0; w0 < g.K; w0 += kMaxBatch) {
+        const int nw = std::min(kMaxBatch, g.K - w0);
+        BatchPtrs gp{};
+        for (int i = 0; i < nw; ++i) gp.dense[i] = static_cast<const char*>(grads) + (int64_t)(w0 + i) * worker_stride_bytes;
+        TRY(enqueue_local(w0, nw, gp, false));
+    }
+    return HPSGD_OK;
+}
+
+int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs)
+{
+    TRY(need_init());
+    if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
+    if (g.K > kMaxBatch) return fail(HPSGD_E_UNSUPPORTED, "batched sparse steps support K <= %d", kMaxBatch);
+    if (!descs) return fail(HPSGD_E_BADARG, "descriptor array is NULL");
+    for (int i = 0; i < g.K; ++i) TRY(check_desc(descs + i));
+    BatchPtrs gp{};
+    TRY(enqueue_slot_maps(0, g.K, descs, &gp));
+    return enqueue_local(0, g.K, gp, true);
+}
+
+int hpsgd_local_step_host(int worker, const void* host_grads)
+{
+    TRY(need_init());
+    TRY(check_worker(worker));
+    if (!host_grads) return fail(HPSGD_E_BADARG, "host_grads is NULL");
+    const size_t bytes = (size_t)g.P_pad * (g.grad_dtype == HPSGD_BF16 ? 2 : 4);
+    if (!g.copy) {
+        CUDA_TRY(cudaStreamCreateWithFlags(&g.copy, cudaStreamNonBlocking));
+        for (int b = 0; b < 2; ++b) {
+            cudaError_t e = cudaMalloc(&g.stage[b], (size_t)g.P_pad * 4);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                return fail(HPSGD_E_NOMEM, "cudaMalloc of the staging buffer failed: %s", cudaGetErrorString(e));
+            }
+            CUDA_TRY(cudaEventCreateWithFlags(&g.stage_copied[b], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&g.stage_free[b], cudaEventDisableTiming));
+        }
+    }
+    const int b = g.stage_next;
+    g.stage_next ^= 1;
+    if (g.stage_used[b]) CUDA_TRY(cudaStreamWaitEvent(g.copy, g.stage_free[b], 0));
+    CUDA_TRY(cudaMemcpyAsync(g.stage[b], host_grads, bytes, cudaMemcpyHostToDevice, g.copy));
+    CUDA_TRY(cudaEventRecord(g.stage_copied[b], g.copy));
+    CUDA_TRY(cudaStreamWaitEvent(g.main, g.stage_copied[b], 0));
+    BatchPtrs gp{};
+    gp.dense[0] = g.stage[b];
+    TRY(enqueue_local(worker, 1, gp, false));
+    CUDA_TRY(cudaEventRecord(g.stage_free[b], g.main));
+    g.stage_used[b] = true;
+    return HPSGD_OK;
+}
+
+// ------------------------------------------------------------------------- merge
+int hpsgd_sync_merge(void)
+{
+    TRY(need_init());
+    cudaStream_t s = g.overlap ? g.side : g.main;
+    int flags = 0;
+    if (g.staleness == 0) flags |= kMergeImmediate;
+    else if (g.D_valid) flags |= kMergeApplyPending;
+    for (int c = 0; c < g.chunks; ++c) {
+        int64_t lo, hi;
+        chunk_range(c, &lo, &hi);
+        if (hi <= lo) continue;
+        if (g.overlap && g.local_recorded[c]) {
+            CUDA_TRY(cudaStreamWaitEvent(s, g.ev_local[c], 0));
+            g.local_recorded[c] = 0;
+        }
+        EventPair ep{};
+        TRY(prof_begin(s, 1, &ep));
+        switch (g.K) {
+        case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
+        case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
+        case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
+        default: launch_merge<0>(s, lo, hi - lo, flags); break;
+        }
+        ++g.launches;
+        TRY(prof_end(s, &ep));
+        if (g.overlap) {
+            CUDA_TRY(cudaEventRecord(g.ev_merge[c], s));
+            g.merge_unwaited[c] = 1;
+        }
+    }
+    g.D_valid = true;
+    g.merges += 1;
+    return check_async();
+}
+
+const float* hpsgd_get_global(void)
+{
+    if (need_init()) return nullptr;
+    if (sync_all()) return nullptr;
+    if (check_async()) return nullptr;
+    return g.w;
+}
+
+// ------------------------------------------------------------------------- host copies, inspection
+int hpsgd_set_global_host(const float* host_w, int64_t n)
+{
+    TRY(need_init());
+    if (!host_w || n != g.P) return fail(HPSGD_E_BADARG, "need a host array of exactly P = %lld floats", (long long)g.P);
+    TRY(sync_all());
+    CUDA_TRY(cudaMemsetAsync(g.w, 0, (size_t)g.stride * 4, g.main));
+    for (size_t t = 0; t < g.sizes.size(); ++t)
+        CUDA_TRY(cudaMemcpyAsync(g.w + g.offsets[t], host_w + g.starts[t], (size_t)g.sizes[t] * 4,
+                                 cudaMemcpyHostToDevice, g.main));
+    return reset_state_from_w();
+}
+
+int hpsgd_copy_global(float* host_out, int64_t n)
+{
+    TRY(need_init());
+    if (!host_out || n != g.P) return fail(HPSGD_E_BADARG, "need a host array of exactly P = %lld floats", (long long)g.P);
+    TRY(sync_all());
+    for (size_t t = 0; t < g.sizes.size(); ++t)
+        CUDA_TRY(cudaMemcpyAsync(host_out + g.starts[t], g.w + g.offsets[t], (size_t)g.sizes[t] * 4,
+                                 cudaMemcpyDeviceToHost, g.main));
+    CUDA_TRY(cudaStreamSynchronize(g.main));
+    return HPSGD_OK;
+}
+
+int hpsgd_get_replica(int worker, const float** r, const float** m)
+{
+    TRY(need_init());
+    TRY(check_worker(worker));
+    if (r) *r = g.r + (int64_t)worker * g.stride;
+    if (m) *m = g.m ? g.m + (int64_t)worker * g.stride : nullptr;
+    return HPSGD_OK;
+}
+
+int hpsgd_get_pending(const float** D)
+{
+    TRY(need_init());
+    if (D) *D = g.D;
+    return HPSGD_OK;
+}
+
+int hpsgd_get_sizes(int64_t* P, int64_t* P_pad, int* K, int64_t* merges)
+{
+    TRY(need_init());
+    if (P) *P = g.P;
+    if (P_pad) *P_pad = g.P_pad;
+    if (K) *K = g.K;
+    if (merges) *merges = g.merges;
+    return HPSGD_OK;
+}
+
+int64_t hpsgd_tensor_offset(int tensor_id)
+{
+    TRY(need_init());
+    if (tensor_id < 0 || tensor_id >= (int)g.sizes.size()) return fail(HPSGD_E_BADARG, "tensor %d does not exist", tensor_id);
+    return g.offsets[tensor_id];
+}
+
+// ------------------------------------------------------------------------- generators
+int hpsgd_gen_grads(void* out, int worker, int step, int kind, double scale)
+{
+    TRY(check_gen_args(out, worker, step, kind));
+    const GenParams gp = gen_params(worker, step, kind, scale);
+    const size_t n = g.sizes.size();
+    if (g.grad_dtype == HPSGD_BF16)
+        gen_flat_kernel<true><<<grid_for(gen_flat_kernel<true>, g.P_pad, kThreads), kThreads, 0, g.main>>>(
+            out, g.P_pad, g.d_table, g.d_table + n, g.d_table + 2 * n, (int)n, gp);
+    else
+        gen_flat_kernel<false><<<grid_for(gen_flat_kernel<false>, g.P_pad, kThreads), kThreads, 0, g.main>>>(
+            out, g.P_pad, g.d_table, g.d_table + n, g.d_table + 2 * n, (int)n, gp);
+    ++g.launches;
+    return check_async();
+}
+
+int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
+                       const int32_t* row_idx, int32_t n_rows)
+{
+    TRY(check_gen_args(out, worker, step, kind));
+    if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
+    if (n_rows < 0 || n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows out of range");
+    if (n_rows == 0) return HPSGD_OK;
+    if (!row_idx) return fail(HPSGD_E_BADARG, "row_idx is NULL");
+    const GenParams gp = gen_params(worker, step, kind, scale);
+    const int64_t n = (int64_t)n_rows * g.sp_cols;
+    if (g.grad_dtype == HPSGD_BF16)
+        gen_rows_kernel<true><<<grid_for(gen_rows_kernel<true>, n, kThreads), kThreads, 0, g.main>>>(out, row_idx, n_rows, gp);
+    else
+        gen_rows_kernel<false><<<grid_for(gen_rows_kernel<false>, n, kThreads), kThreads, 0, g.main>>>(out, row_idx, n_rows, gp);
+    ++g.launches;
+    return check_async();
+}
+
+// ------------------------------------------------------------------------- profiling, counters
+int hpsgd_profile_read(double* local_ms, int64_t* local_launches, double* merge_ms, int64_t* merge_launches)
+{
+    TRY(need_init());
+    TRY(sync_all());
+    TRY(prof_resolve());
+    if (local_ms) *local_ms = g.prof_ms[0];
+    if (local_launches) *local_launches = g.prof_launches[0];
+    if (merge_ms) *merge_ms = g.prof_ms[1];
+    if (merge_launches) *merge_launches = g.prof_launches[1];
+    g.prof_ms[0] = g.prof_ms[1] = 0;
+    g.prof_launches[0] = g.prof_launches[1] = 0;
+    return HPSGD_OK;
+}
+
+int64_t hpsgd_launch_count(void) { return g.inited ? g.launches : 0; }
+
+}  // extern "C"

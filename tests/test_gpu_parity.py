@@ -1,0 +1,225 @@
+"""CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2009_02701_b200 as hp
+import workloads
+from tests import gpu_util as gu
+from tests.oracle_pins import GOLDEN, parse_worked
+from workloads.configs import Workload
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, K, sizes, T=4, lr=0.1, momentum=0.9, wd=0.0, seed=7, kind="gauss", scale=1e-2,
+          dtype="f32", sparse=None, staleness=1):
+    return Workload(name, K=K, sizes=tuple(sizes), T=T, lr=lr, momentum=momentum, weight_decay=wd,
+                    seed=seed, grad_kind=kind, grad_scale=scale, grad_dtype=dtype, sparse=sparse,
+                    staleness=staleness)
+
+
+def test_worked_examples_through_the_abi():
+    """The hand-worked K=2, P=4 rounds (Algorithms 2/3, Eq. 1) reproduced by the kernels."""
+    import os
+    mu, w0, grads, cases = parse_worked(os.path.join(GOLDEN, "worked_k2_p4.txt"))
+    for c in cases:
+        cfg = small("worked", 2, [4], lr=mu, momentum=c["beta"], wd=c["lambda"], staleness=c["staleness"])
+        with gu.session(cfg):
+            hp.hpsgd_set_global_host(np.array(w0, dtype=np.float32))
+            for t in range(3):
+                keep = []
+                for i in range(2):
+                    g = np.zeros(32, dtype=np.float32)
+                    g[:4] = grads[(t, i)]
+                    keep.append(gu.to_device(g))
+                    hp.hpsgd_local_step(i, keep[-1])
+                w, D, rs, ms = gu.gpu_state(cfg)
+                for i in range(2):
+                    np.testing.assert_array_equal(rs[i], np.float32(c["r"][(t, i)]))
+                hp.hpsgd_sync_merge()
+                w, D, rs, ms = gu.gpu_state(cfg)
+                np.testing.assert_array_equal(D, np.float32(c["D"][t]))
+                np.testing.assert_array_equal(w, np.float32(c["w"][t]))
+                np.testing.assert_array_equal(rs[0], w)
+                np.testing.assert_array_equal(rs[1], w)
+
+
+def test_cfg1_full():
+    cfg = workloads.get("cfg1")
+    got, want = gu.run_both(cfg, cfg.T, check_each_round=True)
+    assert gu.max_rel_err(got, want) <= 1e-6
+
+
+@pytest.mark.parametrize("P", [1, 3, 5, 31, 33, 127, 129, 1000, 4097, 70001])
+@pytest.mark.parametrize("K,momentum,wd", [(1, 0.0, 0.0), (2, 0.9, 0.0), (3, 0.9, 5e-4), (5, 0.0, 1e-3),
+                                           (4, 0.9, 0.0), (8, 0.9, 5e-4), (16, 0.9, 0.0), (9, 0.5, 0.0)])
+def test_odd_sizes(P, K, momentum, wd):
+    cfg = small("odd", K, [P], T=3, momentum=momentum, wd=wd)
+    gu.run_both(cfg, cfg.T, check_each_round=(P <= 129))
+
+
+def test_multi_tensor_ragged_layout():
+    rng = np.random.default_rng(5)
+    sizes = [int(x) for x in rng.integers(1, 3000, size=37)] + [64, 32, 1, 33, 100_003]
+    cfg = small("ragged", 6, sizes, T=5, wd=5e-4)
+    gu.run_both(cfg, cfg.T, session_kw=dict(lend_arena=True, canary=True, streams=True))
+
+
+@pytest.mark.parametrize("staleness", [0, 1])
+def test_staleness_modes_and_many_local_steps(staleness):
+    cfg = small("hsteps", 4, [5000, 77], T=4, staleness=staleness)
+    gu.run_both(cfg, cfg.T, staleness=staleness, steps_per_round=3, check_each_round=True)
+
+
+def test_worker_without_a_step_contributes_zero():
+    cfg = small("skip", 4, [3000], T=3)
+    gu.run_both(cfg, cfg.T, skip_worker=2)
+
+
+@pytest.mark.parametrize("overlap,chunks,batched", [(0, 1, False), (1, 1, False), (1, 3, False), (1, 7, True),
+                                                    (0, 5, True), (1, 64, True)])
+def test_schedule_does_not_change_results(overlap, chunks, batched):
+    cfg = small("sched", 8, [300_000, 1234, 99_999], T=6, wd=1e-4)
+    gu.run_both(cfg, cfg.T, overlap=overlap, chunks=chunks, batched=batched)
+
+
+@pytest.mark.parametrize("batched", [False, True])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sparse_rows_and_bf16_small(batched, dtype):
+    # embedding-like [rows x cols] tensor in the middle of the layout, ~10 % rows active
+    cfg = small("sparse", 5, [1000, 300 * 64, 777, 64], T=4, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
+    gu.run_both(cfg, cfg.T, batched=batched, chunks=3)
+
+
+def test_sparse_equals_dense_with_zero_rows():
+    cfg = small("sparse_dense", 3, [128 * 16, 50], T=3, dtype="bf16", sparse=(0, 128, 16), scale=1e-3)
+    results = []
+    for sparse_api in (True, False):
+        with gu.session(cfg):
+            for t in range(cfg.T):
+                keep = []
+                for i in range(cfg.K):
+                    gu.gpu_step(cfg, i, gu.host_inputs(cfg, i, t), keep, sparse_api=sparse_api)
+                hp.hpsgd_sync_merge()
+                hp.hpsgd_synchronize()
+            results.append(gu.gpu_state(cfg))
+    for a, b in zip(results[0][2] + results[0][3] + [results[0][0]], results[1][2] + results[1][3] + [results[1][0]]):
+        gu.assert_bitwise(a, b, "sparse vs dense-with-zero-rows")
+
+
+def test_bf16_gradients_against_fp32_master():
+    """Stored-bf16 gradients vs an oracle fed the un-rounded fp32 gradients: within 1e-2."""
+    cfg = small("bf16master", 4, [50_000], T=10, dtype="bf16", scale=1e-3, lr=0.01)
+    o = gu.oracle_for(cfg)
+    with gu.session(cfg):
+        for t in range(cfg.T):
+            keep = []
+            for i in range(cfg.K):
+                gu.gpu_step(cfg, i, gu.host_inputs(cfg, i, t), keep)
+                o.local_step(i, cfg.gradient(i, t))              # fp32, not rounded to bf16
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+            hp.hpsgd_synchronize()
+        got = gu.gpu_global(cfg)
+    want = o.get_global()
+    # bf16 keeps 8 significand bits: each stored gradient is within 2^-9 of its fp32 value, so
+    # the accumulated change agrees to well under 1e-2 of its size, and each parameter to 1e-2
+    # relative.  Parameters are O(0.1); the denominator is floored at 1e-4 (0.1 % of that
+    # scale) because a parameter that happens to sit at ~1e-6 has no meaningful relative error.
+    assert gu.max_rel_err(got, want, floor=1e-4) <= 1e-2
+    w0 = cfg.initial_global().astype(np.float64)
+    change_err = np.linalg.norm((got - w0) - (want - w0)) / np.linalg.norm(want - w0)
+    assert change_err <= 1e-2
+
+
+def test_device_generator_matches_host_generator():
+    for cfg in (small("gen_u", 3, [1000, 37, 5000], kind="uniform", scale=1e-2, seed=1),
+                small("gen_g", 3, [1000, 37, 5000], kind="gauss", scale=1e-3, seed=2),
+                small("gen_b", 3, [40 * 8, 100, 7], kind="gauss", scale=1e-3, seed=5, dtype="bf16",
+                      sparse=(0, 40, 8))):
+        with gu.session(cfg):
+            gu.assert_bitwise(gu.gpu_global(cfg), cfg.initial_global(), "initial model from the device hash")
+            kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
+            for worker, step in ((0, 0), (2, 9), (1, 1000)):
+                want = cfg.layout.pack(cfg.stored_gradient(worker, step))
+                if cfg.grad_dtype == "bf16":
+                    out = torch.empty(cfg.layout.P_pad, dtype=torch.int16, device=gu.DEV)
+                else:
+                    out = torch.empty(cfg.layout.P_pad, dtype=torch.float32, device=gu.DEV)
+                hp.hpsgd_gen_grads(out, worker, step, kind, cfg.grad_scale)
+                hp.hpsgd_synchronize()
+                got = out.cpu().numpy()
+                if cfg.grad_dtype == "bf16":
+                    got = got.view(np.uint16)
+                    off = np.abs(got.astype(np.int64) - want.astype(np.int64))
+                else:
+                    off = np.abs(got.view(np.int32).astype(np.int64) - want.view(np.int32).astype(np.int64))
+                if cfg.grad_kind == "uniform":
+                    assert off.max() == 0
+                else:
+                    # host and device log/cos may differ in the last binary64 bit
+                    assert off.max() <= 1 and (off > 0).mean() <= 1e-4
+                if cfg.sparse:
+                    rows = cfg.sparse_rows(worker, step)
+                    idx = gu.to_device(rows)
+                    vals = torch.empty(len(rows) * cfg.sparse[2], dtype=torch.int16, device=gu.DEV)
+                    hp.hpsgd_gen_row_vals(vals, worker, step, kind, cfg.grad_scale, idx, len(rows))
+                    hp.hpsgd_synchronize()
+                    wantv = gu.host_inputs(cfg, worker, step)["vals"].reshape(-1)
+                    offv = np.abs(vals.cpu().numpy().view(np.uint16).astype(np.int64) - wantv.astype(np.int64))
+                    assert offv.max() <= 1 and (offv > 0).mean() <= 1e-4
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_resnet_like_configs_full(name):
+    """Full parameter count, every round, every element compared."""
+    cfg = workloads.get(name)
+    got, want = gu.run_both(cfg, cfg.T, batched=(name == "cfg3"), chunks=4)
+    assert gu.max_rel_err(got, want) <= 1e-6
+
+
+def test_host_buffer_entry_point():
+    cfg = small("hostbuf", 3, [200_000, 333], T=3)
+    o = gu.oracle_for(cfg)
+    with gu.session(cfg):
+        pinned = [torch.empty(cfg.layout.P_pad, dtype=torch.float32).pin_memory() for _ in range(cfg.K)]
+        for t in range(cfg.T):
+            for i in range(cfg.K):
+                inp = gu.host_inputs(cfg, i, t)
+                pinned[i].numpy()[:] = inp["padded"]
+                hp.hpsgd_local_step_host(i, pinned[i])
+                o.local_step(i, inp["flat"])
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+            hp.hpsgd_synchronize()
+        gu.assert_bitwise(gu.gpu_global(cfg), o.get_global(), "global via host buffers")
+
+
+def test_argument_errors_enqueue_nothing():
+    cfg = small("errors", 2, [1000], T=1)
+    with gu.session(cfg):
+        before = hp.hpsgd_launch_count()
+        g = torch.zeros(cfg.layout.P_pad + 8, dtype=torch.float32, device=gu.DEV)
+        for call, code in ((lambda: hp.hpsgd_local_step(2, g), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_local_step(-1, g), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_local_step(0, None), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_local_step(0, g.data_ptr() + 4), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_init(10, 2, 0.1, 0.0, 1), hp.HPSGD_E_STATE),
+                           (lambda: hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 0), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_set_option(99, 0), hp.HPSGD_E_BADARG),
+                           (lambda: hp.hpsgd_local_step_ex(0, hp.make_desc(g)), hp.HPSGD_E_STATE),
+                           (lambda: hp.hpsgd_set_sparse_segment(0, 10, 10), hp.HPSGD_E_BADARG)):
+            with pytest.raises(hp.HpsgdError) as err:
+                call()
+            assert err.value.code == code
+        assert hp.hpsgd_launch_count() == before
+    # an arena that is too small is refused before anything is touched
+    hp.hpsgd_destroy()
+    buf = torch.empty(4096, dtype=torch.uint8, device=gu.DEV)
+    base = buf.data_ptr() + (-buf.data_ptr()) % 256
+    hp.hpsgd_bind(base, 1024, None, None)
+    with pytest.raises(hp.HpsgdError) as err:
+        hp.hpsgd_init(100_000, 4, 0.1, 0.9, 1)
+    assert err.value.code == hp.HPSGD_E_NOMEM
+    hp.hpsgd_destroy()
