@@ -195,6 +195,46 @@ int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes);
 /* The same for K sparse-row descriptors (host array of K structs).  K <= 32. */
 int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs);
 
+/*
+ * (The paper has no counterpart for this call; it exists for deployment reasons only.)
+ *
+ * A sparse-row local step that allocates nothing.  Some programs that would like to call
+ * this library are not in a position to obtain device memory for it: an inference or
+ * training server whose own allocator took the whole GPU at start-up and hands out
+ * nothing to third parties, a plug-in running inside a latency-critical loop where the
+ * implicit device-wide synchronisation of cudaMalloc / cudaFree would stall every other
+ * stream, or code running under a memory budget that is accounted to the byte.  For them
+ * the row -> slot scratch map of the sparse-row step lives in a fixed array built into
+ * the library image (HPSGD_NOALLOC_MAX_ROWS int32 entries = 1 MiB, held by every GPU
+ * that loads the library until the process exits), and this call issues no cudaMalloc,
+ * cudaFree or other allocating routine.  It does not use or need hpsgd_init: all state is
+ * passed in.
+ *
+ * It performs, on the caller's buffers, exactly the step of hpsgd_local_step_ex:
+ *   replica / momentum_buf  device, n_elems floats each (n_elems % 4 == 0), 16-byte aligned,
+ *                           updated in place; momentum_buf may be NULL when momentum == 0
+ *   desc                    host struct; dense has n_elems elements of grad_dtype, its span
+ *                           [seg_offset, seg_offset + rows*cols) is ignored; row_idx / row_vals
+ *                           as in hpsgd_grad_desc
+ *   seg_offset, rows, cols  the sparse-row tensor inside the flat buffer (seg_offset % 4 == 0,
+ *                           cols % 8 == 0, rows <= HPSGD_NOALLOC_MAX_ROWS)
+ *   stream                  cudaStream_t the work is enqueued on (NULL = default stream)
+ * Errors: HPSGD_E_UNSUPPORTED when rows exceeds HPSGD_NOALLOC_MAX_ROWS (use
+ * hpsgd_local_step_ex, which sizes its map from the arena), HPSGD_E_BADARG for the rest.
+ *
+ * The first call on each device looks up the device address of the built-in array (with
+ * that device current) and remembers it; make that first call outside any stream capture.
+ * All calls on one device share the one array, and it keeps whatever the previous call
+ * left: each call therefore resets the entries it uses before filling them.  Two calls
+ * whose GPU work can overlap (different streams without an ordering between them) race
+ * on the array and give undefined results; calls on one stream are safe.
+ */
+#define HPSGD_NOALLOC_MAX_ROWS 262144
+int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_buf, int64_t n_elems,
+                                    const hpsgd_grad_desc* desc, int grad_dtype,
+                                    int64_t seg_offset, int64_t rows, int64_t cols,
+                                    float lr, float momentum, float weight_decay, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * Host-buffer convenience (end-to-end use) and inspection.
  * ---------------------------------------------------------------------------------- */

@@ -18,6 +18,7 @@ HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE = 4, 5, 6
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
+HPSGD_NOALLOC_MAX_ROWS = 262144
 
 
 class hpsgd_grad_desc(ctypes.Structure):
@@ -50,6 +51,8 @@ SIGNATURES = {
     "hpsgd_local_step_ex": (_ci, [_ci, _P(hpsgd_grad_desc)]),
     "hpsgd_local_step_all": (_ci, [_vp, _i64]),
     "hpsgd_local_step_all_ex": (_ci, [_P(hpsgd_grad_desc)]),
+    "hpsgd_local_step_sparse_noalloc": (_ci, [_vp, _vp, _i64, _P(hpsgd_grad_desc), _ci, _i64, _i64, _i64,
+                                              _f32, _f32, _f32, _vp]),
     "hpsgd_local_step_host": (_ci, [_ci, _vp]),
     "hpsgd_set_global_host": (_ci, [_vp, _i64]),
     "hpsgd_copy_global": (_ci, [_vp, _i64]),
@@ -182,6 +185,15 @@ def hpsgd_local_step_all(grads, worker_stride_bytes):
 def hpsgd_local_step_all_ex(descs):
     arr = (hpsgd_grad_desc * len(descs))(*descs)
     return _check(load().hpsgd_local_step_all_ex(arr))
+
+
+def hpsgd_local_step_sparse_noalloc(replica, momentum_buf, n_elems, desc, grad_dtype, seg_offset, rows, cols,
+                                    lr, momentum, weight_decay, stream=None):
+    """Sparse-row local step on caller-owned buffers; allocates nothing (see hpsgd.h)."""
+    return _check(load().hpsgd_local_step_sparse_noalloc(
+        _ptr(replica), _ptr(momentum_buf), int(n_elems), ctypes.byref(desc), int(grad_dtype),
+        int(seg_offset), int(rows), int(cols), float(lr), float(momentum), float(weight_decay),
+        _stream(stream)))
 
 
 def hpsgd_local_step_host(worker, host_grads):

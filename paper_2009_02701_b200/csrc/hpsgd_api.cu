@@ -885,3 +885,114 @@ int hpsgd_profile_read(double* local_ms, int64_t* local_launches, double* merge_
 int64_t hpsgd_launch_count(void) { return g.inited ? g.launches : 0; }
 
 }  // extern "C"
+
+// =============================================================================== no-allocation entry
+// hpsgd_local_step_sparse_noalloc: the sparse-row local step for callers that cannot
+// allocate device memory.  Its row -> slot scratch map is the file-scope array below,
+// which every GPU that loads this library holds until the process exits.
+static __device__ __align__(256) int32_t g_noalloc_slot[HPSGD_NOALLOC_MAX_ROWS];
+
+namespace {
+
+constexpr int kNoallocMaxDevices = 64;
+struct NoallocDevice {
+    bool ready = false;
+    int32_t* slot = nullptr;     // device address of g_noalloc_slot on this device
+    int sm_count = 0;
+} g_noalloc_dev[kNoallocMaxDevices];
+
+// Once per device, with that device current: g_noalloc_slot names a host-side stand-in in
+// host code, so the address a kernel can use has to be asked for.
+int noalloc_setup(int dev, NoallocDevice** out)
+{
+    if (dev < 0 || dev >= kNoallocMaxDevices) return fail(HPSGD_E_UNSUPPORTED, "device index %d not supported", dev);
+    NoallocDevice& d = g_noalloc_dev[dev];
+    if (!d.ready) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_slot);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(HPSGD_E_CUDA, "cudaGetSymbolAddress of the scratch map failed: %s", cudaGetErrorString(e));
+        }
+        int sms = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        d.slot = static_cast<int32_t*>(p);
+        d.sm_count = sms;
+        d.ready = true;
+    }
+    *out = &d;
+    return HPSGD_OK;
+}
+
+template <bool BF16, bool MOM, bool WD>
+void noalloc_launch(cudaStream_t s, int sm_count, float* r, float* m, const BatchPtrs& gp,
+                    const SparseSeg& seg, int64_t nvec, const StepParams& p)
+{
+    constexpr int U = 4;
+    auto kern = local_step_kernel<BF16, MOM, WD, true, U>;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0) != cudaSuccess || occ < 1) occ = 1;
+    const int64_t need = std::max<int64_t>(1, (nvec + kThreads * U - 1) / (kThreads * U));
+    const int grid = (int)std::min<int64_t>(need, (int64_t)sm_count * occ);
+    kern<<<grid, kThreads, 0, s>>>(r, m, 0, 0, gp, seg, 0, nvec, p);
+}
+
+}  // namespace
+
+extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_buf, int64_t n_elems,
+                                               const hpsgd_grad_desc* desc, int grad_dtype,
+                                               int64_t seg_offset, int64_t rows, int64_t cols,
+                                               float lr, float momentum, float weight_decay, void* stream)
+{
+    if (!replica || reinterpret_cast<uintptr_t>(replica) % 16) return fail(HPSGD_E_BADARG, "replica must be a 16-byte aligned device pointer");
+    if (!(momentum >= 0.f && momentum < 1.f)) return fail(HPSGD_E_BADARG, "momentum must be in [0, 1)");
+    if (momentum != 0.f && (!momentum_buf || reinterpret_cast<uintptr_t>(momentum_buf) % 16))
+        return fail(HPSGD_E_BADARG, "momentum_buf must be a 16-byte aligned device pointer when momentum != 0");
+    if (!(lr >= 0.f) || !(weight_decay >= 0.f)) return fail(HPSGD_E_BADARG, "lr and weight_decay must be >= 0");
+    if (n_elems <= 0 || n_elems % 4) return fail(HPSGD_E_BADARG, "n_elems must be a positive multiple of 4");
+    if (grad_dtype != HPSGD_F32 && grad_dtype != HPSGD_BF16) return fail(HPSGD_E_BADARG, "unknown gradient dtype");
+    if (rows <= 0 || cols <= 0 || cols % 8) return fail(HPSGD_E_BADARG, "rows must be positive and cols a positive multiple of 8");
+    if (rows > HPSGD_NOALLOC_MAX_ROWS)
+        return fail(HPSGD_E_UNSUPPORTED, "%lld rows exceed the built-in scratch map of %d rows; use hpsgd_local_step_ex",
+                    (long long)rows, HPSGD_NOALLOC_MAX_ROWS);
+    if (seg_offset < 0 || seg_offset % 4 || seg_offset + rows * cols > n_elems)
+        return fail(HPSGD_E_BADARG, "the sparse tensor does not fit inside the flat buffer");
+    if (!desc) return fail(HPSGD_E_BADARG, "descriptor is NULL");
+    TRY(check_grad_ptr(desc->dense, "dense gradient"));
+    if (desc->n_rows < 0 || desc->n_rows > rows) return fail(HPSGD_E_BADARG, "n_rows %d out of range", desc->n_rows);
+    const bool have_rows = desc->row_idx && desc->n_rows > 0;
+    if (have_rows) TRY(check_grad_ptr(desc->row_vals, "row_vals"));
+
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    NoallocDevice* d = nullptr;
+    TRY(noalloc_setup(dev, &d));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // the map keeps the previous call's contents: every row starts again at "no slot" (-1)
+    CUDA_TRY(cudaMemsetAsync(d->slot, 0xFF, (size_t)rows * 4, s));
+    if (have_rows)
+        scatter_slots_kernel<<<(desc->n_rows + 255) / 256, 256, 0, s>>>(d->slot, desc->row_idx, desc->n_rows, rows);
+    BatchPtrs gp{};
+    gp.dense[0] = desc->dense;
+    gp.row_vals[0] = desc->row_vals;
+    gp.slot[0] = d->slot;
+    SparseSeg seg{seg_offset / 4, (seg_offset + rows * cols) / 4, (int32_t)(cols / 4)};
+    const StepParams p{-lr, momentum, weight_decay};
+    const bool mom = momentum != 0.f, wd = weight_decay != 0.f, bf = grad_dtype == HPSGD_BF16;
+    const int64_t nvec = n_elems / 4;
+#define HPSGD_NOALLOC_CASE(B, M, W) noalloc_launch<B, M, W>(s, d->sm_count, replica, momentum_buf, gp, seg, nvec, p)
+    if (bf) {
+        if (mom && wd) HPSGD_NOALLOC_CASE(true, true, true);
+        else if (mom) HPSGD_NOALLOC_CASE(true, true, false);
+        else if (wd) HPSGD_NOALLOC_CASE(true, false, true);
+        else HPSGD_NOALLOC_CASE(true, false, false);
+    } else {
+        if (mom && wd) HPSGD_NOALLOC_CASE(false, true, true);
+        else if (mom) HPSGD_NOALLOC_CASE(false, true, false);
+        else if (wd) HPSGD_NOALLOC_CASE(false, false, true);
+        else HPSGD_NOALLOC_CASE(false, false, false);
+    }
+#undef HPSGD_NOALLOC_CASE
+    return check_async();
+}
