@@ -325,7 +325,7 @@ def run_gpu(args, cfg):
 
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step
     e2e = None
-    if rank == 0 or dist is not None:
+    if args.e2e_steps > 0:
         e2e = run_e2e(args, cfg, hp, torch, dev, grads, dist)
 
     line = None

@@ -91,7 +91,7 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed);
  *     gd = g + lambda*r_i ;  m_i = beta*m_i + gd ;  r_i = r_i - mu*m_i
  * each line one fused multiply-add in binary32, round to nearest even.  `grads` is a
  * device buffer of P_pad elements in the flat layout, fp32 or bf16 per
- * HPSGD_OPT_GRAD_DTYPE, 16-byte aligned, zero in the pads.  It is borrowed: keep it
+ * HPSGD_OPT_GRAD_DTYPE, 32-byte aligned, zero in the pads.  It is borrowed: keep it
  * valid and unchanged until the work has run (hpsgd_synchronize, or a stream wait on
  * the main stream).  Several local steps per worker between two merges are legal
  * (Section 3.2: several local trainings per synchronisation); a worker with none
@@ -161,7 +161,7 @@ int hpsgd_set_option(int key, double value);
  * hpsgd_local_step; inside the span of the sparse tensor its contents are ignored.
  * The sparse tensor (declared by hpsgd_set_sparse_segment) is [rows x cols]; row_idx
  * (device, int32, ascending, unique, each in [0, rows)) lists the n_rows rows that carry
- * a gradient and row_vals (device, [n_rows x cols], same dtype as dense, 16-byte
+ * a gradient and row_vals (device, [n_rows x cols], same dtype as dense, 32-byte
  * aligned) their values.  Rows not listed have gradient ZERO and are still stepped
  * (momentum decays and moves the replica, weight decay applies): the result equals
  * a dense step with zero rows.  row_idx == NULL or n_rows == 0 means no sparse tensor
@@ -185,7 +185,7 @@ int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc);
 
 /*
  * One local step of ALL K workers in one launch per index range: worker i reads its
- * dense gradient at (char*)grads + i * worker_stride_bytes (16-byte aligned stride).
+ * dense gradient at (char*)grads + i * worker_stride_bytes (stride a multiple of 32 bytes).
  * Same arithmetic as K calls of hpsgd_local_step; the launches are issued range by
  * range so that, with HPSGD_OPT_CHUNKS > 1, the merge of a range can start while later
  * ranges are still being stepped.
@@ -211,12 +211,12 @@ int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs);
  * passed in.
  *
  * It performs, on the caller's buffers, exactly the step of hpsgd_local_step_ex:
- *   replica / momentum_buf  device, n_elems floats each (n_elems % 4 == 0), 16-byte aligned,
+ *   replica / momentum_buf  device, n_elems floats each (n_elems % 8 == 0), 32-byte aligned,
  *                           updated in place; momentum_buf may be NULL when momentum == 0
  *   desc                    host struct; dense has n_elems elements of grad_dtype, its span
  *                           [seg_offset, seg_offset + rows*cols) is ignored; row_idx / row_vals
  *                           as in hpsgd_grad_desc
- *   seg_offset, rows, cols  the sparse-row tensor inside the flat buffer (seg_offset % 4 == 0,
+ *   seg_offset, rows, cols  the sparse-row tensor inside the flat buffer (seg_offset % 8 == 0,
  *                           cols % 8 == 0, rows <= HPSGD_NOALLOC_MAX_ROWS)
  *   stream                  cudaStream_t the work is enqueued on (NULL = default stream)
  * Errors: HPSGD_E_UNSUPPORTED when rows exceeds HPSGD_NOALLOC_MAX_ROWS (use

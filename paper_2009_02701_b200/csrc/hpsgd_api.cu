@@ -19,7 +19,8 @@ constexpr int64_t kRowAlignElems = 64;     // rows of r / m: multiples of 256 by
 constexpr size_t kAlignBytes = 256;        // arena regions
 constexpr int kMaxChunks = 1024;
 constexpr int kMaxTensors = 4096;
-constexpr int64_t kChunkGrainVec = 2048;   // chunk boundaries: multiples of 8192 elements
+constexpr int64_t kChunkGrain = 1024;      // chunk boundaries: multiples of 1024 groups (8192 elements)
+constexpr int kMaxGridX = 0x7FFFFFFF;
 
 char g_err[512] = "";
 
@@ -134,17 +135,23 @@ ArenaPlan plan_arena(int64_t stride, int K, bool momentum)
     return a;
 }
 
-// Index range [v_lo, v_hi), in 4-element vectors, of schedule chunk c.
-void chunk_range(int c, int64_t* v_lo, int64_t* v_hi)
+// Index range [o_lo, o_hi), in 8-element groups, of schedule chunk c.
+void chunk_range(int c, int64_t* o_lo, int64_t* o_hi)
 {
-    const int64_t nvec = g.P_pad / 4;
-    const int64_t grains = (nvec + kChunkGrainVec - 1) / kChunkGrainVec;
-    auto edge = [&](int k) { return std::min(nvec, grains * k / g.chunks * kChunkGrainVec); };
-    *v_lo = edge(c);
-    *v_hi = (c == g.chunks - 1) ? nvec : edge(c + 1);
+    const int64_t n = g.P_pad / 8;
+    const int64_t grains = (n + kChunkGrain - 1) / kChunkGrain;
+    auto edge = [&](int k) { return std::min(n, grains * k / g.chunks * kChunkGrain); };
+    *o_lo = edge(c);
+    *o_hi = (c == g.chunks - 1) ? n : edge(c + 1);
 }
 
-// Grid: enough blocks to cover `items` at `per_block` each, capped at one full wave of
+// Grid of the hot kernels: one block per kHotThreads groups.
+int hot_grid(int64_t groups)
+{
+    return (int)std::min<int64_t>(kMaxGridX, std::max<int64_t>(1, (groups + kHotThreads - 1) / kHotThreads));
+}
+
+// Grid of the support kernels: enough blocks to cover `items`, capped at one full wave of
 // resident blocks (SM count x blocks the kernel can keep resident per SM).
 template <typename Kern>
 int grid_for(Kern kern, int64_t items, int64_t per_block)
@@ -194,17 +201,16 @@ struct LocalLaunch {
     int w0, nw;
     BatchPtrs gp;
     SparseSeg seg;
-    int64_t v0, nvec;
+    int64_t o0, n;
     StepParams p;
 };
 
 template <bool BF16, bool MOM, bool WD, bool SPARSE>
 void launch_local(const LocalLaunch& L)
 {
-    constexpr int U = 4;
-    auto kern = local_step_kernel<BF16, MOM, WD, SPARSE, U>;
-    dim3 grid(grid_for(kern, L.nvec, (int64_t)kThreads * U), L.nw);
-    kern<<<grid, kThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.v0, L.nvec, L.p);
+    dim3 grid(hot_grid(L.n), L.nw);
+    local_step_kernel<BF16, MOM, WD, SPARSE><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp,
+                                                                               L.seg, L.o0, L.n, L.p);
 }
 
 template <bool BF16, bool MOM, bool WD>
@@ -231,9 +237,9 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
     L.p = StepParams{-g.lr, g.beta, g.lambda};
     L.seg = SparseSeg{0, 0, 1};
     if (sparse) {
-        L.seg.v_begin = g.offsets[g.sp_tensor] / 4;
-        L.seg.v_end = L.seg.v_begin + g.sp_rows * g.sp_cols / 4;
-        L.seg.cols4 = (int32_t)(g.sp_cols / 4);
+        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
+        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
+        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
     }
     const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
     for (int c = 0; c < g.chunks; ++c) {
@@ -244,7 +250,7 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
             CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
             g.merge_unwaited[c] = 0;
         }
-        L.v0 = lo; L.nvec = hi - lo;
+        L.o0 = lo; L.n = hi - lo;
         EventPair ep{};
         TRY(prof_begin(g.main, 0, &ep));
         if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
@@ -280,7 +286,7 @@ int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* g
 int check_grad_ptr(const void* p, const char* what)
 {
     if (!p) return fail(HPSGD_E_BADARG, "%s is NULL", what);
-    if (reinterpret_cast<uintptr_t>(p) % 16) return fail(HPSGD_E_BADARG, "%s is not 16-byte aligned", what);
+    if (reinterpret_cast<uintptr_t>(p) % 32) return fail(HPSGD_E_BADARG, "%s is not 32-byte aligned", what);
     return HPSGD_OK;
 }
 
@@ -398,10 +404,9 @@ void release_all()
 }
 
 template <int KT>
-void launch_merge(cudaStream_t s, int64_t v0, int64_t nvec, int flags)
+void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
 {
-    auto kern = merge_kernel<KT>;
-    kern<<<grid_for(kern, nvec, kThreads), kThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, v0, nvec, flags);
+    merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags);
 }
 
 }  // namespace
@@ -676,8 +681,8 @@ int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes)
     TRY(need_init());
     TRY(check_grad_ptr(grads, "grads"));
     const int64_t esz = g.grad_dtype == HPSGD_BF16 ? 2 : 4;
-    if (worker_stride_bytes % 16 || worker_stride_bytes < g.P_pad * esz)
-        return fail(HPSGD_E_BADARG, "worker stride must be a multiple of 16 bytes and cover P_pad elements");
+    if (worker_stride_bytes % 32 || worker_stride_bytes < g.P_pad * esz)
+        return fail(HPSGD_E_BADARG, "worker stride must be a multiple of 32 bytes and cover P_pad elements");
     for (int w0 = 0; w0 < g.K; w0 += kMaxBatch) {
         const int nw = std::min(kMaxBatch, g.K - w0);
         BatchPtrs gp{};
@@ -926,15 +931,10 @@ int noalloc_setup(int dev, NoallocDevice** out)
 
 template <bool BF16, bool MOM, bool WD>
 void noalloc_launch(cudaStream_t s, int sm_count, float* r, float* m, const BatchPtrs& gp,
-                    const SparseSeg& seg, int64_t nvec, const StepParams& p)
+                    const SparseSeg& seg, int64_t n, const StepParams& p)
 {
-    constexpr int U = 4;
-    auto kern = local_step_kernel<BF16, MOM, WD, true, U>;
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0) != cudaSuccess || occ < 1) occ = 1;
-    const int64_t need = std::max<int64_t>(1, (nvec + kThreads * U - 1) / (kThreads * U));
-    const int grid = (int)std::min<int64_t>(need, (int64_t)sm_count * occ);
-    kern<<<grid, kThreads, 0, s>>>(r, m, 0, 0, gp, seg, 0, nvec, p);
+    (void)sm_count;
+    local_step_kernel<BF16, MOM, WD, true><<<hot_grid(n), kHotThreads, 0, s>>>(r, m, 0, 0, gp, seg, 0, n, p);
 }
 
 }  // namespace
@@ -944,18 +944,18 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
                                                int64_t seg_offset, int64_t rows, int64_t cols,
                                                float lr, float momentum, float weight_decay, void* stream)
 {
-    if (!replica || reinterpret_cast<uintptr_t>(replica) % 16) return fail(HPSGD_E_BADARG, "replica must be a 16-byte aligned device pointer");
+    if (!replica || reinterpret_cast<uintptr_t>(replica) % 32) return fail(HPSGD_E_BADARG, "replica must be a 32-byte aligned device pointer");
     if (!(momentum >= 0.f && momentum < 1.f)) return fail(HPSGD_E_BADARG, "momentum must be in [0, 1)");
-    if (momentum != 0.f && (!momentum_buf || reinterpret_cast<uintptr_t>(momentum_buf) % 16))
-        return fail(HPSGD_E_BADARG, "momentum_buf must be a 16-byte aligned device pointer when momentum != 0");
+    if (momentum != 0.f && (!momentum_buf || reinterpret_cast<uintptr_t>(momentum_buf) % 32))
+        return fail(HPSGD_E_BADARG, "momentum_buf must be a 32-byte aligned device pointer when momentum != 0");
     if (!(lr >= 0.f) || !(weight_decay >= 0.f)) return fail(HPSGD_E_BADARG, "lr and weight_decay must be >= 0");
-    if (n_elems <= 0 || n_elems % 4) return fail(HPSGD_E_BADARG, "n_elems must be a positive multiple of 4");
+    if (n_elems <= 0 || n_elems % 8) return fail(HPSGD_E_BADARG, "n_elems must be a positive multiple of 8");
     if (grad_dtype != HPSGD_F32 && grad_dtype != HPSGD_BF16) return fail(HPSGD_E_BADARG, "unknown gradient dtype");
     if (rows <= 0 || cols <= 0 || cols % 8) return fail(HPSGD_E_BADARG, "rows must be positive and cols a positive multiple of 8");
     if (rows > HPSGD_NOALLOC_MAX_ROWS)
         return fail(HPSGD_E_UNSUPPORTED, "%lld rows exceed the built-in scratch map of %d rows; use hpsgd_local_step_ex",
                     (long long)rows, HPSGD_NOALLOC_MAX_ROWS);
-    if (seg_offset < 0 || seg_offset % 4 || seg_offset + rows * cols > n_elems)
+    if (seg_offset < 0 || seg_offset % 8 || seg_offset + rows * cols > n_elems)
         return fail(HPSGD_E_BADARG, "the sparse tensor does not fit inside the flat buffer");
     if (!desc) return fail(HPSGD_E_BADARG, "descriptor is NULL");
     TRY(check_grad_ptr(desc->dense, "dense gradient"));
@@ -977,10 +977,10 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
     gp.dense[0] = desc->dense;
     gp.row_vals[0] = desc->row_vals;
     gp.slot[0] = d->slot;
-    SparseSeg seg{seg_offset / 4, (seg_offset + rows * cols) / 4, (int32_t)(cols / 4)};
+    SparseSeg seg{seg_offset / 8, (seg_offset + rows * cols) / 8, (int32_t)(cols / 8)};
     const StepParams p{-lr, momentum, weight_decay};
     const bool mom = momentum != 0.f, wd = weight_decay != 0.f, bf = grad_dtype == HPSGD_BF16;
-    const int64_t nvec = n_elems / 4;
+    const int64_t nvec = n_elems / 8;
 #define HPSGD_NOALLOC_CASE(B, M, W) noalloc_launch<B, M, W>(s, d->sm_count, replica, momentum_buf, gp, seg, nvec, p)
     if (bf) {
         if (mom && wd) HPSGD_NOALLOC_CASE(true, true, true);
