@@ -18,6 +18,7 @@ path has no inter-GPU exchange); time is the max over ranks, value the sum of un
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -60,29 +61,37 @@ def merge_bytes_per_index(cfg):
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """nvidia-smi clock / throttle-reason samples; only those taken inside the timed window
+    (host wall clock between mark_begin and mark_end) are summarised."""
 
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index):
         self.gpu_index = gpu_index
         self.proc = None
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
+    def mark_begin(self):
+        self.t0 = datetime.datetime.now()
+
+    def mark_end(self):
+        self.t1 = datetime.datetime.now()
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
@@ -91,11 +100,16 @@ class ClockSampler:
             out, _ = self.proc.communicate()
         sm, smax, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        total = 0
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
+            total += 1
             try:
+                stamp = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+                if self.t0 and self.t1 and not (self.t0 <= stamp <= self.t1):
+                    continue
                 sm.append(float(f[1]))
                 smax.append(float(f[2]))
                 power.append(float(f[3]))
@@ -107,7 +121,7 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
                 "power_w_max": max(power) if power else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples_in_timed_region": len(sm), "samples_total": total, "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------ CPU oracle legs
@@ -270,7 +284,11 @@ def run_gpu(args, cfg):
             hp.hpsgd_local_step_all(grads[b], P_pad * gsz)
         hp.hpsgd_sync_merge()
 
-    # ---- warm-up, then the timed region
+    # ---- warm-up, then the timed region (the clock sampler needs a moment to start)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
     for t in range(args.warmup):
         one_round(t)
     hp.hpsgd_synchronize()
@@ -279,9 +297,7 @@ def run_gpu(args, cfg):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(dev)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
+    sampler.mark_begin()
     launches0 = hp.hpsgd_launch_count()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record(main)
@@ -290,6 +306,7 @@ def run_gpu(args, cfg):
     main.wait_stream(side)
     end.record(main)
     torch.cuda.synchronize(dev)
+    sampler.mark_end()
     if dist is not None:
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
@@ -401,7 +418,7 @@ def run_e2e(args, cfg, hp, torch, dev, grads, dist):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=workloads.names())

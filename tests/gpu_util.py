@@ -229,3 +229,21 @@ def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, batched=False, step
     want = o.get_global()
     o.close()
     return got, want
+
+
+def dev_gather(addr: int, n: int, positions: np.ndarray) -> np.ndarray:
+    """Elements at `positions` of the n-float device buffer at a raw address."""
+    view = torch.as_tensor(_RawDeviceArray(addr, n, "<f4"), device=DEV)
+    return view[torch.from_numpy(np.ascontiguousarray(positions, dtype=np.int64)).to(DEV)].cpu().numpy()
+
+
+def stratified_sample(cfg, n_random=1 << 18, edge=64, seed=12345) -> np.ndarray:
+    """Un-padded indices: the first and last `edge` elements of every tensor plus random ones."""
+    picks = []
+    for size, start in zip(cfg.layout.sizes, cfg.layout.starts):
+        e = min(edge, size)
+        picks.append(np.arange(start, start + e))
+        picks.append(np.arange(start + size - e, start + size))
+    rng = np.random.default_rng(seed)
+    picks.append(rng.integers(0, cfg.P, size=n_random))
+    return np.unique(np.concatenate(picks)).astype(np.int64)

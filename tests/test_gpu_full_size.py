@@ -1,0 +1,80 @@
+"""Full-size workloads (cfg4: 138M parameters x 16 workers, cfg5: GRU-shaped, bf16 + sparse
+rows) in the launch configuration the benchmark times: gradients generated on the device,
+one batched local-step call and one merge per round.  The oracle cannot run 2.2 G
+parameters x T rounds in seconds, and every index is independent of every other, so it
+recomputes a stratified sample of indices (both ends of every tensor plus 2^18 random
+ones) from the HOST generator and those are compared."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2009_02701_b200 as hp
+import workloads
+from oracle.ref import RefHPSGD
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def run_full(cfg, T):
+    lay = cfg.layout
+    K, P_pad = cfg.K, lay.P_pad
+    bf16 = cfg.grad_dtype == "bf16"
+    gdt = torch.int16 if bf16 else torch.float32
+    kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
+    idx = gu.stratified_sample(cfg)
+    pos = lay.padded_index(idx)
+
+    oracle = RefHPSGD(idx.size, K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+    oracle.set_global(cfg.initial_global(idx))
+
+    with gu.session(cfg, lend_arena=True, streams=True, canary=True):
+        grads = torch.empty((K, P_pad), dtype=gdt, device=gu.DEV)
+        for t in range(T):
+            hp.hpsgd_synchronize()                   # the one gradient buffer is reused every round
+            descs, keep = [], []
+            for i in range(K):
+                hp.hpsgd_gen_grads(grads[i], i, t, kind, cfg.grad_scale)
+                if cfg.sparse:
+                    rows = gu.to_device(cfg.sparse_rows(i, t))
+                    vals = torch.empty(rows.numel() * cfg.sparse[2], dtype=gdt, device=gu.DEV)
+                    hp.hpsgd_gen_row_vals(vals, i, t, kind, cfg.grad_scale, rows, rows.numel())
+                    keep += [rows, vals]
+                    descs.append(hp.make_desc(grads[i], rows, rows.numel(), vals))
+            if cfg.sparse:
+                hp.hpsgd_local_step_all_ex(descs)
+            else:
+                hp.hpsgd_local_step_all(grads, P_pad * grads.element_size())
+            hp.hpsgd_sync_merge()
+            for i in range(K):
+                oracle.local_step(i, cfg.stored_gradient(i, t, idx))
+            oracle.sync_merge()
+        hp.hpsgd_synchronize()
+        got = {"w": gu.dev_gather(hp.hpsgd_get_global(), P_pad, pos),
+               "D": gu.dev_gather(hp.hpsgd_get_pending(), P_pad, pos)}
+        for i in (0, K // 2, K - 1):
+            r, m = hp.hpsgd_get_replica(i)
+            got["r%d" % i] = gu.dev_gather(r, P_pad, pos)
+            got["m%d" % i] = gu.dev_gather(m, P_pad, pos)
+    want = {"w": oracle.get_global(), "D": oracle.get_pending()}
+    for i in (0, K // 2, K - 1):
+        want["r%d" % i] = oracle.get_replica(i)
+        want["m%d" % i] = oracle.get_momentum(i)
+    oracle.close()
+    return idx, got, want
+
+
+@pytest.mark.parametrize("name", ["cfg4", "cfg5"])
+def test_full_size_sampled_parity(name):
+    cfg = workloads.get(name)
+    idx, got, want = run_full(cfg, cfg.T)
+    assert idx.size > 250_000
+    for key in got:
+        # parameters and replicas to 1e-6 relative (floor 1e-6); the momentum and pending-change
+        # buffers are compared at the scale of the quantity they hold
+        floor = 1e-6 if key[0] in "wr" else 1e-9
+        err = gu.max_rel_err(got[key], want[key], floor=floor)
+        assert err <= 1e-6, "%s: max relative error %g" % (key, err)
+        equal = np.mean(got[key].view(np.uint32) == want[key].view(np.uint32))
+        # device and host log/cos may round a Gaussian differently once in ~1e8 draws
+        assert equal >= 0.999, "%s: only %.6f of the sample is bit-equal" % (key, equal)
