@@ -55,6 +55,29 @@ def local_bytes_per_elem(cfg):
     return g + 8 + (8 if cfg.momentum else 0)
 
 
+def fused_bytes_per_index(cfg):
+    """Fused merge + local step: the merge without its K replica writes plus the K local steps
+    without their replica reads = 16 + K * (local step bytes)."""
+    return 16 + cfg.K * local_bytes_per_elem(cfg)
+
+
+# DRAM bytes per parameter index (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture divided by the indices of that launch), keyed by (kernel, K, gradient dtype), with
+# the SHA-1 of the kernel source the capture was taken from.  A changed source voids them.
+NCU_TRAFFIC = {}
+
+
+def ncu_traffic(kernel, cfg, algorithmic_bytes_per_launch):
+    entry = NCU_TRAFFIC.get((kernel, cfg.K, cfg.grad_dtype))
+    if entry is None:
+        return None
+    import hashlib
+    src = os.path.join(ROOT, "paper_2009_02701_b200", "csrc", "hpsgd_kernels.cuh")
+    if hashlib.sha1(open(src, "rb").read()).hexdigest() != entry["source_sha1"]:
+        return None
+    return entry["bytes_per_index"] * cfg.P
+
+
 def merge_bytes_per_index(cfg):
     """Algorithmic HBM bytes per parameter index of one merge: (2K + 4) * 4."""
     return (2 * cfg.K + 4) * 4
@@ -243,6 +266,7 @@ def run_gpu(args, cfg):
     hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
     hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
     hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, args.chunks)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, args.fuse)
     if cfg.sparse:
         hp.hpsgd_set_sparse_segment(*cfg.sparse)
 
@@ -292,8 +316,9 @@ def run_gpu(args, cfg):
     for t in range(args.warmup):
         one_round(t)
     hp.hpsgd_synchronize()
-    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)
-    hp.hpsgd_profile_read()
+    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)     # also launches a merge deferred by the warm-up
+    for kind in range(3):
+        hp.hpsgd_profile_read(kind)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(dev)
@@ -303,6 +328,7 @@ def run_gpu(args, cfg):
     start.record(main)
     for t in range(args.steps):
         one_round(args.warmup + t)
+    hp.hpsgd_flush()                                 # the last round's merge, if it was deferred
     main.wait_stream(side)
     end.record(main)
     torch.cuda.synchronize(dev)
@@ -312,33 +338,40 @@ def run_gpu(args, cfg):
     clocks = sampler.stop() if rank == 0 else None
     elapsed_ms = start.elapsed_time(end)
     launches = hp.hpsgd_launch_count() - launches0
-    local_ms, local_n, merge_ms, merge_n = hp.hpsgd_profile_read()
+    prof = {name: hp.hpsgd_profile_read(kind) for kind, name in
+            enumerate(("local_step_kernel", "merge_kernel", "merge_step_kernel"))}
     hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 0)
     units = K * P * args.steps
     job_ms, job_units = aggregate(dist, dev, elapsed_ms, units)
     value = job_units / (job_ms * 1e-3)
 
-    # ---- roofline of the two kernels from the event pairs recorded inside the timed region
+    # ---- roofline of the kernels from the event pairs recorded inside the timed region.
+    # Algorithmic bytes per launch = bytes per parameter index x indices one launch covers.
     peak, peak_src = measured_peak()
-    merge_launch_bytes = merge_bytes_per_index(cfg) * P * args.steps / max(merge_n, 1)
-    local_launch_bytes = local_bytes_per_elem(cfg) * P * K * args.steps / max(local_n, 1)
-    merge_gbs = merge_bytes_per_index(cfg) * P * args.steps / (merge_ms * 1e-3) / 1e9 if merge_ms else 0.0
-    local_gbs = local_bytes_per_elem(cfg) * P * K * args.steps / (local_ms * 1e-3) / 1e9 if local_ms else 0.0
-    kernels = {
-        "merge_kernel": {"launches": merge_n, "avg_ms": merge_ms / max(merge_n, 1), "algorithmic_bytes_per_launch": merge_launch_bytes,
-                         "achieved": merge_gbs, "frac": merge_gbs / peak, "frac_of_nominal_8TBs": merge_gbs / NOMINAL_HBM_GBS},
-        "local_step_kernel": {"launches": local_n, "avg_ms": local_ms / max(local_n, 1), "algorithmic_bytes_per_launch": local_launch_bytes,
-                              "achieved": local_gbs, "frac": local_gbs / peak, "frac_of_nominal_8TBs": local_gbs / NOMINAL_HBM_GBS},
-    }
-    dominant = "local_step_kernel" if local_ms >= merge_ms else "merge_kernel"
+    per_index = {"local_step_kernel": local_bytes_per_elem(cfg) * (1 if args.per_worker else K),
+                 "merge_kernel": merge_bytes_per_index(cfg),
+                 "merge_step_kernel": fused_bytes_per_index(cfg)}
+    kernels = {}
+    for name, (ms, n) in prof.items():
+        if n == 0:
+            continue
+        per_launch = per_index[name] * P / args.chunks
+        gbs = per_launch * n / (ms * 1e-3) / 1e9
+        kernels[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms, "algorithmic_bytes_per_launch": per_launch,
+                         "achieved": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+    dominant = max(kernels, key=lambda k: kernels[k]["total_ms"])
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved"], "peak": peak,
-                "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": None,
+                "unit": "GB/s", "frac": kernels[dominant]["frac"],
+                "traffic": ncu_traffic(dominant, cfg, kernels[dominant]["algorithmic_bytes_per_launch"]),
                 "peak_source": peak_src, "nominal_peak": NOMINAL_HBM_GBS, "kernels": kernels,
-                "note": "event pairs around each launch on its own stream inside the timed region; "
-                        "with chunks > 1 the two kernels overlap and share HBM"}
-    round_bytes = (local_bytes_per_elem(cfg) * K + merge_bytes_per_index(cfg)) * P
-    roofline["round_achieved"] = round_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
+                "note": "CUDA event pairs around each launch on its own stream inside the timed region; "
+                        "a fused merge_step_kernel launch moves 16 + K*(local step bytes) per index, "
+                        "8K fewer than the merge and local-step launches it replaces"}
+    moved = sum(k["algorithmic_bytes_per_launch"] * k["launches"] for k in kernels.values())
+    roofline["round_achieved"] = moved / (elapsed_ms * 1e-3) / 1e9
     roofline["round_frac"] = roofline["round_achieved"] / peak
+    unfused_round = (local_bytes_per_elem(cfg) * K + merge_bytes_per_index(cfg)) * P
+    roofline["round_unfused_equivalent"] = unfused_round * args.steps / (elapsed_ms * 1e-3) / 1e9
 
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step
     e2e = None
@@ -358,7 +391,7 @@ def run_gpu(args, cfg):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic (counter-hash gradients generated on the device, %d rounds cycled)" % nbuf,
             "config": workload_config(cfg, {
-                "schedule": {"overlap": args.overlap, "chunks": args.chunks,
+                "schedule": {"overlap": args.overlap, "chunks": args.chunks, "fuse_merge_into_next_step": args.fuse,
                              "local_step_call": "per worker" if args.per_worker else "all K in one call"},
                 "l2": "inputs larger than L2 (state + gradients are tens of GB)",
                 "multi_gpu": "independent replicas, no inter-GPU exchange"}),
@@ -424,6 +457,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=workloads.names())
     ap.add_argument("--overlap", type=int, default=1)
     ap.add_argument("--chunks", type=int, default=1)
+    ap.add_argument("--fuse", type=int, default=1, help="carry each merge into the next batched local step (one kernel)")
     ap.add_argument("--per-worker", action="store_true", help="K hpsgd_local_step calls instead of one batched call")
     ap.add_argument("--grad-buffers", type=int, default=2, help="rounds of device-resident gradients to cycle")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -55,9 +55,18 @@ enum {
                                    steps by events; 0: everything on the main stream. */
     HPSGD_OPT_CHUNKS = 5,       /* number of index ranges the schedule is cut into (1..1024).
                                    Results do not depend on it. Default 1. */
-    HPSGD_OPT_PROFILE = 6       /* 1: bracket every local-step call and every merge with CUDA
-                                   events on the stream it runs on (see hpsgd_profile_read). */
+    HPSGD_OPT_PROFILE = 6,      /* 1: bracket every kernel launch of the path with CUDA events
+                                   on the stream it runs on (see hpsgd_profile_read). */
+    HPSGD_OPT_FUSE = 7          /* 1: hpsgd_sync_merge does not launch its merge at once; if the next
+                                   call is a batched local step (hpsgd_local_step_all[_ex], K <= 32)
+                                   both run as ONE kernel in which the re-cloned replica never goes
+                                   to memory; any other call first launches the merge on its own.
+                                   Same operations in the same order: results are bit-identical.
+                                   Default 0. */
 };
+
+/* Kernel kinds of hpsgd_profile_read. */
+enum { HPSGD_KERNEL_LOCAL_STEP = 0, HPSGD_KERNEL_MERGE = 1, HPSGD_KERNEL_MERGE_STEP = 2 };
 
 enum { HPSGD_F32 = 0, HPSGD_BF16 = 1 };
 
@@ -108,7 +117,8 @@ int hpsgd_local_step(int worker, const void* grads);
  *     r_i  = w  for every i
  * in one fused kernel.  m_i is not touched.  Enqueued on the side stream (main stream
  * when HPSGD_OPT_OVERLAP is 0) behind all local steps issued so far; later local steps
- * wait, per index range, for the part of the merge they depend on.
+ * wait, per index range, for the part of the merge they depend on.  With HPSGD_OPT_FUSE
+ * the launch is deferred to the next call (see that option); the result is the same.
  */
 int hpsgd_sync_merge(void);
 
@@ -303,13 +313,16 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
 int hpsgd_synchronize(void);
 
 /*
- * With HPSGD_OPT_PROFILE on: total device milliseconds and number of kernel launches of
- * the local-step kernels and of the merge kernels since the last read, measured with
- * CUDA event pairs recorded around each launch on the stream it ran on.  Synchronises
- * and resets the totals.  Any out pointer may be NULL.
+ * With HPSGD_OPT_PROFILE on: total device milliseconds and number of launches of one kind
+ * of kernel (HPSGD_KERNEL_*: local step, merge, fused merge + local step) since the last
+ * read of that kind, measured with CUDA event pairs recorded around each launch on the
+ * stream it ran on.  Launches any deferred merge, synchronises, and resets that kind's
+ * totals.  Any out pointer may be NULL.
  */
-int hpsgd_profile_read(double* local_ms, int64_t* local_launches,
-                       double* merge_ms, int64_t* merge_launches);
+int hpsgd_profile_read(int kind, double* ms, int64_t* launches);
+
+/* Enqueue a merge that HPSGD_OPT_FUSE deferred, if there is one (does not wait). */
+int hpsgd_flush(void);
 
 /* Number of kernels this library has launched since hpsgd_init. */
 int64_t hpsgd_launch_count(void);

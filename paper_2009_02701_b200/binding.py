@@ -14,7 +14,8 @@ HPSGD_OK = 0
 HPSGD_E_BADARG, HPSGD_E_STATE, HPSGD_E_NOMEM = -1, -2, -3
 HPSGD_E_CUDA, HPSGD_E_TIMEOUT, HPSGD_E_UNSUPPORTED = -4, -5, -6
 HPSGD_OPT_WEIGHT_DECAY, HPSGD_OPT_STALENESS, HPSGD_OPT_GRAD_DTYPE = 1, 2, 3
-HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE = 4, 5, 6
+HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE, HPSGD_OPT_FUSE = 4, 5, 6, 7
+HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP = 0, 1, 2
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
@@ -63,7 +64,8 @@ SIGNATURES = {
     "hpsgd_gen_grads": (_ci, [_vp, _ci, _ci, _ci, _f64]),
     "hpsgd_gen_row_vals": (_ci, [_vp, _ci, _ci, _ci, _f64, _vp, ctypes.c_int32]),
     "hpsgd_synchronize": (_ci, []),
-    "hpsgd_profile_read": (_ci, [_P(_f64), _P(_i64), _P(_f64), _P(_i64)]),
+    "hpsgd_profile_read": (_ci, [_ci, _P(_f64), _P(_i64)]),
+    "hpsgd_flush": (_ci, []),
     "hpsgd_launch_count": (_i64, []),
     "hpsgd_last_error": (ctypes.c_char_p, []),
     "hpsgd_destroy": (_ci, []),
@@ -248,11 +250,15 @@ def hpsgd_synchronize():
     return _check(load().hpsgd_synchronize())
 
 
-def hpsgd_profile_read():
-    """Returns (local_ms, local_launches, merge_ms, merge_launches) since the last read."""
-    a, b, c, d = _f64(), _i64(), _f64(), _i64()
-    _check(load().hpsgd_profile_read(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(d)))
-    return a.value, b.value, c.value, d.value
+def hpsgd_profile_read(kind):
+    """Returns (milliseconds, launches) of one kernel kind since its last read."""
+    ms, n = _f64(), _i64()
+    _check(load().hpsgd_profile_read(int(kind), ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value
+
+
+def hpsgd_flush():
+    return _check(load().hpsgd_flush())
 
 
 def hpsgd_launch_count():

@@ -50,7 +50,7 @@ size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct EventPair {
     cudaEvent_t a, b;
-    int kind;       // 0 local step, 1 merge
+    int kind;       // HPSGD_KERNEL_*
 };
 
 struct Pending {                // configuration collected before hpsgd_init
@@ -83,6 +83,9 @@ struct Ctx {
     std::vector<char> local_recorded, merge_unwaited;
     bool D_valid = false;
     int64_t merges = 0;
+    int fuse = 0;                          // carry a merge into the next batched local step
+    bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
+    int deferred_flags = 0;
     int64_t launches = 0;
     int sm_count = 148;
     int sp_tensor = -1;                    // sparse-row tensor
@@ -92,8 +95,8 @@ struct Ctx {
     bool stage_used[2] = {false, false};
     int stage_next = 0;
     std::vector<EventPair> prof;           // profiling
-    double prof_ms[2] = {0, 0};
-    int64_t prof_launches[2] = {0, 0};
+    double prof_ms[3] = {0, 0, 0};
+    int64_t prof_launches[3] = {0, 0, 0};
 } g;
 
 int check_async()
@@ -252,7 +255,7 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
         }
         L.o0 = lo; L.n = hi - lo;
         EventPair ep{};
-        TRY(prof_begin(g.main, 0, &ep));
+        TRY(prof_begin(g.main, HPSGD_KERNEL_LOCAL_STEP, &ep));
         if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
         else launch_local_d<false>(mom, wd, sparse, L);
         ++g.launches;
@@ -407,6 +410,123 @@ template <int KT>
 void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
 {
     merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags);
+}
+
+// Enqueue one merge, chunk by chunk, on the side stream (main stream without overlap).
+int enqueue_merge(int flags)
+{
+    cudaStream_t s = g.overlap ? g.side : g.main;
+    for (int c = 0; c < g.chunks; ++c) {
+        int64_t lo, hi;
+        chunk_range(c, &lo, &hi);
+        if (hi <= lo) continue;
+        if (g.overlap && g.local_recorded[c]) {
+            CUDA_TRY(cudaStreamWaitEvent(s, g.ev_local[c], 0));
+            g.local_recorded[c] = 0;
+        }
+        EventPair ep{};
+        TRY(prof_begin(s, HPSGD_KERNEL_MERGE, &ep));
+        switch (g.K) {
+        case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
+        case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
+        case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
+        default: launch_merge<0>(s, lo, hi - lo, flags); break;
+        }
+        ++g.launches;
+        TRY(prof_end(s, &ep));
+        if (g.overlap) {
+            CUDA_TRY(cudaEventRecord(g.ev_merge[c], s));
+            g.merge_unwaited[c] = 1;
+        }
+    }
+    return check_async();
+}
+
+// A merge that hpsgd_sync_merge deferred (fuse option) and that nothing has absorbed yet.
+int flush_deferred()
+{
+    if (!g.merge_deferred) return HPSGD_OK;
+    g.merge_deferred = false;
+    return enqueue_merge(g.deferred_flags);
+}
+
+struct FusedLaunch {
+    BatchPtrs gp;
+    SparseSeg seg;
+    int64_t o0, n;
+    int flags;
+    StepParams p;
+};
+
+template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
+void launch_fused(const FusedLaunch& L)
+{
+    merge_step_kernel<KT, BF16, MOM, WD, SPARSE><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
+        g.w, g.D, g.r, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p);
+}
+
+template <int KT, bool BF16>
+void launch_fused_d(bool mom, bool wd, bool sparse, const FusedLaunch& L)
+{
+#define HPSGD_FUSED_CASE(M, W)                                    \
+    do {                                                          \
+        if (sparse) launch_fused<KT, BF16, M, W, true>(L);        \
+        else launch_fused<KT, BF16, M, W, false>(L);              \
+    } while (0)
+    if (mom && wd) HPSGD_FUSED_CASE(true, true);
+    else if (mom) HPSGD_FUSED_CASE(true, false);
+    else if (wd) HPSGD_FUSED_CASE(false, true);
+    else HPSGD_FUSED_CASE(false, false);
+#undef HPSGD_FUSED_CASE
+}
+
+template <bool BF16>
+void launch_fused_k(bool mom, bool wd, bool sparse, const FusedLaunch& L)
+{
+    switch (g.K) {
+    case 4: launch_fused_d<4, BF16>(mom, wd, sparse, L); break;
+    case 8: launch_fused_d<8, BF16>(mom, wd, sparse, L); break;
+    case 16: launch_fused_d<16, BF16>(mom, wd, sparse, L); break;
+    default: launch_fused_d<0, BF16>(mom, wd, sparse, L); break;
+    }
+}
+
+// The deferred merge and the local step of all K workers in one kernel per chunk (main stream).
+int enqueue_fused(const BatchPtrs& gp, bool sparse)
+{
+    FusedLaunch L{};
+    L.gp = gp;
+    L.flags = g.deferred_flags;
+    L.p = StepParams{-g.lr, g.beta, g.lambda};
+    L.seg = SparseSeg{0, 0, 1};
+    if (sparse) {
+        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
+        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
+        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
+    }
+    g.merge_deferred = false;
+    const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
+    for (int c = 0; c < g.chunks; ++c) {
+        int64_t lo, hi;
+        chunk_range(c, &lo, &hi);
+        if (hi <= lo) continue;
+        if (g.merge_unwaited[c]) {
+            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
+            g.merge_unwaited[c] = 0;
+        }
+        L.o0 = lo; L.n = hi - lo;
+        EventPair ep{};
+        TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE_STEP, &ep));
+        if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
+        else launch_fused_k<false>(mom, wd, sparse, L);
+        ++g.launches;
+        TRY(prof_end(g.main, &ep));
+        if (g.overlap) {
+            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
+            g.local_recorded[c] = 1;
+        }
+    }
+    return check_async();
 }
 
 }  // namespace
@@ -573,6 +693,7 @@ int hpsgd_destroy(void)
 int hpsgd_synchronize(void)
 {
     TRY(need_init());
+    TRY(flush_deferred());
     TRY(sync_all());
     return check_async();
 }
@@ -580,6 +701,7 @@ int hpsgd_synchronize(void)
 int hpsgd_set_option(int key, double value)
 {
     TRY(need_init());
+    TRY(flush_deferred());
     switch (key) {
     case HPSGD_OPT_WEIGHT_DECAY:
         if (!(value >= 0.0)) return fail(HPSGD_E_BADARG, "weight decay must be >= 0");
@@ -606,6 +728,10 @@ int hpsgd_set_option(int key, double value)
             return fail(HPSGD_E_BADARG, "chunks must be an integer in [1, %d]", kMaxChunks);
         TRY(sync_all());
         return make_chunk_events((int)value);
+    case HPSGD_OPT_FUSE:
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "fuse must be 0 or 1");
+        g.fuse = (int)value;
+        return HPSGD_OK;
     case HPSGD_OPT_PROFILE:
         if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "profile must be 0 or 1");
         TRY(prof_resolve());
@@ -619,6 +745,7 @@ int hpsgd_set_option(int key, double value)
 int hpsgd_set_sparse_segment(int tensor_id, int64_t rows, int64_t cols)
 {
     TRY(need_init());
+    TRY(flush_deferred());
     if (tensor_id < 0) {
         g.sp_tensor = -1;
         g.sp_rows = g.sp_cols = 0;
@@ -660,6 +787,7 @@ int hpsgd_local_step(int worker, const void* grads)
     TRY(need_init());
     TRY(check_worker(worker));
     TRY(check_grad_ptr(grads, "grads"));
+    TRY(flush_deferred());
     BatchPtrs gp{};
     gp.dense[0] = grads;
     return enqueue_local(worker, 1, gp, false);
@@ -671,6 +799,7 @@ int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc)
     TRY(check_worker(worker));
     if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
     TRY(check_desc(desc));
+    TRY(flush_deferred());
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(worker, 1, desc, &gp));
     return enqueue_local(worker, 1, gp, true);
@@ -683,6 +812,12 @@ int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes)
     const int64_t esz = g.grad_dtype == HPSGD_BF16 ? 2 : 4;
     if (worker_stride_bytes % 32 || worker_stride_bytes < g.P_pad * esz)
         return fail(HPSGD_E_BADARG, "worker stride must be a multiple of 32 bytes and cover P_pad elements");
+    if (g.merge_deferred && g.K <= kMaxBatch) {
+        BatchPtrs gp{};
+        for (int i = 0; i < g.K; ++i) gp.dense[i] = static_cast<const char*>(grads) + (int64_t)i * worker_stride_bytes;
+        return enqueue_fused(gp, false);
+    }
+    TRY(flush_deferred());
     for (int w0 = 0; w0 < g.K; w0 += kMaxBatch) {
         const int nw = std::min(kMaxBatch, g.K - w0);
         BatchPtrs gp{};
@@ -701,6 +836,7 @@ int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs)
     for (int i = 0; i < g.K; ++i) TRY(check_desc(descs + i));
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(0, g.K, descs, &gp));
+    if (g.merge_deferred) return enqueue_fused(gp, true);
     return enqueue_local(0, g.K, gp, true);
 }
 
@@ -709,6 +845,7 @@ int hpsgd_local_step_host(int worker, const void* host_grads)
     TRY(need_init());
     TRY(check_worker(worker));
     if (!host_grads) return fail(HPSGD_E_BADARG, "host_grads is NULL");
+    TRY(flush_deferred());
     const size_t bytes = (size_t)g.P_pad * (g.grad_dtype == HPSGD_BF16 ? 2 : 4);
     if (!g.copy) {
         CUDA_TRY(cudaStreamCreateWithFlags(&g.copy, cudaStreamNonBlocking));
@@ -740,41 +877,30 @@ int hpsgd_local_step_host(int worker, const void* host_grads)
 int hpsgd_sync_merge(void)
 {
     TRY(need_init());
-    cudaStream_t s = g.overlap ? g.side : g.main;
+    TRY(flush_deferred());                 // two merges in a row: the earlier one runs on its own
     int flags = 0;
     if (g.staleness == 0) flags |= kMergeImmediate;
     else if (g.D_valid) flags |= kMergeApplyPending;
-    for (int c = 0; c < g.chunks; ++c) {
-        int64_t lo, hi;
-        chunk_range(c, &lo, &hi);
-        if (hi <= lo) continue;
-        if (g.overlap && g.local_recorded[c]) {
-            CUDA_TRY(cudaStreamWaitEvent(s, g.ev_local[c], 0));
-            g.local_recorded[c] = 0;
-        }
-        EventPair ep{};
-        TRY(prof_begin(s, 1, &ep));
-        switch (g.K) {
-        case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
-        case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
-        case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
-        default: launch_merge<0>(s, lo, hi - lo, flags); break;
-        }
-        ++g.launches;
-        TRY(prof_end(s, &ep));
-        if (g.overlap) {
-            CUDA_TRY(cudaEventRecord(g.ev_merge[c], s));
-            g.merge_unwaited[c] = 1;
-        }
-    }
     g.D_valid = true;
     g.merges += 1;
-    return check_async();
+    if (g.fuse) {
+        g.merge_deferred = true;
+        g.deferred_flags = flags;
+        return HPSGD_OK;
+    }
+    return enqueue_merge(flags);
+}
+
+int hpsgd_flush(void)
+{
+    TRY(need_init());
+    return flush_deferred();
 }
 
 const float* hpsgd_get_global(void)
 {
     if (need_init()) return nullptr;
+    if (flush_deferred()) return nullptr;
     if (sync_all()) return nullptr;
     if (check_async()) return nullptr;
     return g.w;
@@ -785,6 +911,7 @@ int hpsgd_set_global_host(const float* host_w, int64_t n)
 {
     TRY(need_init());
     if (!host_w || n != g.P) return fail(HPSGD_E_BADARG, "need a host array of exactly P = %lld floats", (long long)g.P);
+    TRY(flush_deferred());
     TRY(sync_all());
     CUDA_TRY(cudaMemsetAsync(g.w, 0, (size_t)g.stride * 4, g.main));
     for (size_t t = 0; t < g.sizes.size(); ++t)
@@ -797,6 +924,7 @@ int hpsgd_copy_global(float* host_out, int64_t n)
 {
     TRY(need_init());
     if (!host_out || n != g.P) return fail(HPSGD_E_BADARG, "need a host array of exactly P = %lld floats", (long long)g.P);
+    TRY(flush_deferred());
     TRY(sync_all());
     for (size_t t = 0; t < g.sizes.size(); ++t)
         CUDA_TRY(cudaMemcpyAsync(host_out + g.starts[t], g.w + g.offsets[t], (size_t)g.sizes[t] * 4,
@@ -873,17 +1001,17 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
 }
 
 // ------------------------------------------------------------------------- profiling, counters
-int hpsgd_profile_read(double* local_ms, int64_t* local_launches, double* merge_ms, int64_t* merge_launches)
+int hpsgd_profile_read(int kind, double* ms, int64_t* launches)
 {
     TRY(need_init());
+    if (kind < 0 || kind > 2) return fail(HPSGD_E_BADARG, "unknown kernel kind %d", kind);
+    TRY(flush_deferred());
     TRY(sync_all());
     TRY(prof_resolve());
-    if (local_ms) *local_ms = g.prof_ms[0];
-    if (local_launches) *local_launches = g.prof_launches[0];
-    if (merge_ms) *merge_ms = g.prof_ms[1];
-    if (merge_launches) *merge_launches = g.prof_launches[1];
-    g.prof_ms[0] = g.prof_ms[1] = 0;
-    g.prof_launches[0] = g.prof_launches[1] = 0;
+    if (ms) *ms = g.prof_ms[kind];
+    if (launches) *launches = g.prof_launches[kind];
+    g.prof_ms[kind] = 0;
+    g.prof_launches[kind] = 0;
     return HPSGD_OK;
 }
 

@@ -232,6 +232,119 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
     }
 }
 
+// ---------------------------------------------------------------------------- merge + next local step
+// The merge followed by the first local step of every worker, in one pass: the clone
+// r_i = w never goes to memory, it is the starting point of r_i - mu*m_i directly
+// (Algorithm 2 makes the replica and updates it in consecutive lines).  Same operations,
+// same order, same results as merge_kernel followed by local_step_kernel, but per index
+// it moves (K r + w + D) in, (w + D) out, then per worker (g + m) in, (r + m) out:
+// (5K + 4) * 4 bytes with fp32 gradients instead of (7K + 4) * 4.
+template <bool BF16, bool SPARSE>
+__device__ __forceinline__ f8 fused_grad8(const BatchPtrs& gp, const SparseSeg& seg, int i, int64_t o)
+{
+    if (SPARSE) {
+        if (o >= seg.o_begin && o < seg.o_end) {
+            const int64_t rel = o - seg.o_begin;
+            const int64_t row = rel / seg.cols8;
+            const int32_t s = __ldg(gp.slot[i] + row);
+            if (s < 0) return zero8();
+            return load_grad8<BF16>(gp.row_vals[i], (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
+        }
+    }
+    return load_grad8<BF16>(gp.dense[i], o);
+}
+
+template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
+__global__ void __launch_bounds__(kHotThreads, 2)
+merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r, float* __restrict__ m,
+                  int64_t stride, int K, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags,
+                  StepParams p)
+{
+    constexpr int B = 4;                         // workers whose g / m are in flight together
+    const int Kn = KT > 0 ? KT : K;
+    const float fK = (float)Kn;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        const int64_t e = o * 8;
+        // ---- merge
+        const f8 wv = ld8(w + e);
+        f8 dv = zero8();
+        if (flags & kMergeApplyPending) dv = ld8(D + e);
+        f8 acc;
+        if constexpr (KT > 0) {
+            f8 rv[KT];
+#pragma unroll
+            for (int i = 0; i < KT; ++i) rv[i] = ld8(r + (int64_t)i * stride + e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(rv[0].v[q], wv.v[q]);
+#pragma unroll
+            for (int i = 1; i < KT; ++i)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
+        } else {
+            {
+                const f8 r0 = ld8(r + e);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
+            }
+            int i = 1;
+            for (; i + 4 <= K; i += 4) {
+                f8 rv[4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) rv[b] = ld8(r + (int64_t)(i + b) * stride + e);
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
+            }
+            for (; i < K; ++i) {
+                const f8 ri = ld8(r + (int64_t)i * stride + e);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
+            }
+        }
+        f8 dnew, wn;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            dnew.v[q] = __fdiv_rn(acc.v[q], fK);
+            wn.v[q] = wv.v[q];
+            if (flags & kMergeImmediate) wn.v[q] = __fadd_rn(wv.v[q], dnew.v[q]);
+            else if (flags & kMergeApplyPending) wn.v[q] = __fadd_rn(wv.v[q], dv.v[q]);
+        }
+        st8(w + e, wn);
+        st8(D + e, dnew);
+        // ---- local step of every worker, starting from the clone r_i = wn
+        int i0 = 0;
+#pragma unroll
+        for (; i0 + B <= Kn; i0 += B) {
+            f8 gg[B], mm[B];
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                gg[b] = fused_grad8<BF16, SPARSE>(gp, seg, i0 + b, o);
+                if (MOM) mm[b] = ld8(m + (int64_t)(i0 + b) * stride + e);
+            }
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                f8 rr;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) rr.v[q] = step1<MOM, WD>(gg[b].v[q], mm[b].v[q], wn.v[q], p);
+                st8(r + (int64_t)(i0 + b) * stride + e, rr);
+                if (MOM) st8(m + (int64_t)(i0 + b) * stride + e, mm[b]);
+            }
+        }
+        for (; i0 < Kn; ++i0) {
+            f8 gg = fused_grad8<BF16, SPARSE>(gp, seg, i0, o);
+            f8 mm;
+            if (MOM) mm = ld8(m + (int64_t)i0 * stride + e);
+            f8 rr;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) rr.v[q] = step1<MOM, WD>(gg.v[q], mm.v[q], wn.v[q], p);
+            st8(r + (int64_t)i0 * stride + e, rr);
+            if (MOM) st8(m + (int64_t)i0 * stride + e, mm);
+        }
+    }
+}
+
 // r_i = w for every worker (used when the state is (re)initialised).
 __global__ void __launch_bounds__(kThreads)
 clone_kernel(const float* __restrict__ w_, float* __restrict__ r_, int64_t stride, int K, int64_t nvec)

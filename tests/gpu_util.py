@@ -35,7 +35,7 @@ def to_device(a: np.ndarray) -> torch.Tensor:
 
 
 @contextlib.contextmanager
-def session(cfg, *, staleness=None, overlap=1, chunks=1, lend_arena=False, streams=False, canary=False):
+def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, lend_arena=False, streams=False, canary=False):
     """hpsgd_init for a workload (layout, options, optional lent arena/streams); destroys on exit."""
     hp.hpsgd_destroy()
     lay = cfg.layout
@@ -65,6 +65,7 @@ def session(cfg, *, staleness=None, overlap=1, chunks=1, lend_arena=False, strea
         hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if cfg.grad_dtype == "bf16" else hp.HPSGD_F32)
         hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, overlap)
         hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, chunks)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
         if cfg.sparse:
             hp.hpsgd_set_sparse_segment(*cfg.sparse)
         yield keep
@@ -174,13 +175,14 @@ def max_rel_err(got, want, floor=1e-6):
     return float(np.max(np.abs(got - want) / np.maximum(np.abs(want), floor)))
 
 
-def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, batched=False, steps_per_round=1,
+def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, fuse=0, batched=False, steps_per_round=1,
              skip_worker=None, session_kw=None, check_each_round=False):
     """Run T rounds on the GPU and on the oracle with host-generated inputs; compare bitwise."""
     o = oracle_for(cfg, staleness)
-    with session(cfg, staleness=staleness, overlap=overlap, chunks=chunks, **(session_kw or {})):
+    with session(cfg, staleness=staleness, overlap=overlap, chunks=chunks, fuse=fuse, **(session_kw or {})):
         assert_bitwise(gpu_global(cfg), o.get_global(), "initial global model")
         step = 0
+        alive = []
         for t in range(T):
             keep = []
             for h in range(steps_per_round):
@@ -215,8 +217,11 @@ def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, batched=False, step
                 w, D, rs, ms = gpu_state(cfg)
                 assert_bitwise(w, o.get_global(), "global after merge %d" % t)
                 assert_bitwise(D, o.get_pending(), "pending change after merge %d" % t)
-            hp.hpsgd_synchronize()
-            del keep
+            if fuse:
+                alive.append(keep)          # no synchronise here: it would launch the deferred merge
+            else:
+                hp.hpsgd_synchronize()
+                del keep
         w, D, rs, ms = gpu_state(cfg)
         assert_bitwise(w, o.get_global(), "global model")
         assert_bitwise(D, o.get_pending(), "pending change")

@@ -223,3 +223,61 @@ def test_argument_errors_enqueue_nothing():
         hp.hpsgd_init(100_000, 4, 0.1, 0.9, 1)
     assert err.value.code == hp.HPSGD_E_NOMEM
     hp.hpsgd_destroy()
+
+
+# ---------------------------------------------------------------- merge fused into the next local step
+@pytest.mark.parametrize("K,momentum,wd,staleness", [(16, 0.9, 0.0, 1), (8, 0.9, 5e-4, 1), (4, 0.0, 0.0, 1),
+                                                      (3, 0.9, 0.0, 1), (5, 0.0, 1e-3, 0), (9, 0.5, 0.0, 1),
+                                                      (1, 0.9, 0.0, 0), (16, 0.9, 1e-4, 0)])
+def test_fused_merge_step_matches_oracle(K, momentum, wd, staleness):
+    cfg = small("fused", K, [70_001, 33, 4096], T=5, momentum=momentum, wd=wd, staleness=staleness)
+    got, want = gu.run_both(cfg, cfg.T, staleness=staleness, fuse=1, batched=True, chunks=3)
+    assert gu.max_rel_err(got, want) <= 1e-6
+
+
+def test_fused_launches_one_kernel_per_round():
+    cfg = small("fused_count", 8, [50_000], T=4)
+    with gu.session(cfg, fuse=1):
+        stacked = np.stack([gu.host_inputs(cfg, i, 0)["padded"] for i in range(cfg.K)])
+        g = gu.to_device(stacked.reshape(-1))
+        hp.hpsgd_local_step_all(g, stacked.shape[1] * 4)
+        hp.hpsgd_sync_merge()
+        hp.hpsgd_synchronize()                       # launches that merge on its own
+        base = hp.hpsgd_launch_count()
+        for t in range(4):
+            hp.hpsgd_local_step_all(g, stacked.shape[1] * 4)
+            hp.hpsgd_sync_merge()
+        assert hp.hpsgd_launch_count() - base == 4  # 1 local step, then 3 fused merge+step kernels
+        hp.hpsgd_flush()
+        assert hp.hpsgd_launch_count() - base == 5  # the last merge
+        hp.hpsgd_flush()
+        assert hp.hpsgd_launch_count() - base == 5
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_fused_sparse_rows(dtype):
+    cfg = small("fused_sparse", 5, [1000, 300 * 64, 777, 64], T=5, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
+    gu.run_both(cfg, cfg.T, fuse=1, batched=True, chunks=2)
+
+
+def test_fused_mixed_with_other_calls():
+    """Per-worker steps, several steps per round and back-to-back merges all force the
+    deferred merge out on its own; the results stay those of the oracle."""
+    cfg = small("fused_mixed", 4, [30_000, 17], T=3, wd=1e-4)
+    gu.run_both(cfg, cfg.T, fuse=1, batched=False)                        # never fuses
+    gu.run_both(cfg, cfg.T, fuse=1, batched=True, steps_per_round=3)      # first step of a round fuses
+    o = gu.oracle_for(cfg)
+    with gu.session(cfg, fuse=1):
+        keep = []
+        for t in range(3):
+            for i in range(cfg.K):
+                inp = gu.host_inputs(cfg, i, t)
+                gu.gpu_step(cfg, i, inp, keep)
+                o.local_step(i, inp["flat"])
+            hp.hpsgd_sync_merge()
+            hp.hpsgd_sync_merge()                                         # a merge with no step in between
+            o.sync_merge()
+            o.sync_merge()
+        w, D, rs, ms = gu.gpu_state(cfg)
+        gu.assert_bitwise(w, o.get_global(), "global after back-to-back merges")
+        gu.assert_bitwise(D, o.get_pending(), "pending change after back-to-back merges")
