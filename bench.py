@@ -348,14 +348,22 @@ def run_gpu(args, cfg):
     # ---- roofline of the kernels from the event pairs recorded inside the timed region.
     # Algorithmic bytes per launch = bytes per parameter index x indices one launch covers.
     peak, peak_src = measured_peak()
-    per_index = {"local_step_kernel": local_bytes_per_elem(cfg) * (1 if args.per_worker else K),
-                 "merge_kernel": merge_bytes_per_index(cfg),
-                 "merge_step_kernel": fused_bytes_per_index(cfg)}
+    # gradient bytes of one round: dense buffers, minus the rows of a sparse-row tensor that carry
+    # no gradient (never read), plus 4 bytes per listed row index
+    grad_bytes = K * P * gsz
+    if cfg.sparse:
+        rows_total, cols = cfg.sparse[1], cfg.sparse[2]
+        active = sum(pw[0].numel() for b in sparse_in for pw in b) / nbuf
+        grad_bytes += active * 4 - (K * rows_total - active) * cols * gsz
+    state_bytes = K * P * (8 + (8 if cfg.momentum else 0))        # r (and m) read and written
+    per_round = {"local_step_kernel": grad_bytes + state_bytes,
+                 "merge_kernel": merge_bytes_per_index(cfg) * P,
+                 "merge_step_kernel": 16 * P + grad_bytes + state_bytes}
     kernels = {}
     for name, (ms, n) in prof.items():
         if n == 0:
             continue
-        per_launch = per_index[name] * P / args.chunks
+        per_launch = per_round[name] / args.chunks / (K if (args.per_worker and name == "local_step_kernel") else 1)
         gbs = per_launch * n / (ms * 1e-3) / 1e9
         kernels[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms, "algorithmic_bytes_per_launch": per_launch,
                          "achieved": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
@@ -370,7 +378,7 @@ def run_gpu(args, cfg):
     moved = sum(k["algorithmic_bytes_per_launch"] * k["launches"] for k in kernels.values())
     roofline["round_achieved"] = moved / (elapsed_ms * 1e-3) / 1e9
     roofline["round_frac"] = roofline["round_achieved"] / peak
-    unfused_round = (local_bytes_per_elem(cfg) * K + merge_bytes_per_index(cfg)) * P
+    unfused_round = per_round["local_step_kernel"] + per_round["merge_kernel"]
     roofline["round_unfused_equivalent"] = unfused_round * args.steps / (elapsed_ms * 1e-3) / 1e9
 
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step

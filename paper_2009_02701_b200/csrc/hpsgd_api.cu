@@ -268,20 +268,27 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
     return check_async();
 }
 
-// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors.
+// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors: one memset over
+// the nw consecutive maps (every row: no slot, -1) and one scatter launch for all of them.
 int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* gp)
 {
+    int32_t* first = g.slot + (int64_t)w0 * g.slot_cap;
+    CUDA_TRY(cudaMemsetAsync(first, 0xFF, (size_t)g.slot_cap * 4 * nw, g.main));
+    SlotBatch sb{};
+    int32_t most = 0;
     for (int i = 0; i < nw; ++i) {
-        int32_t* slot = g.slot + (int64_t)(w0 + i) * g.slot_cap;
-        CUDA_TRY(cudaMemsetAsync(slot, 0xFF, (size_t)g.sp_rows * 4, g.main));     // every row: no slot (-1)
         const hpsgd_grad_desc& d = descs[i];
-        if (d.row_idx && d.n_rows > 0) {
-            scatter_slots_kernel<<<(d.n_rows + 255) / 256, 256, 0, g.main>>>(slot, d.row_idx, d.n_rows, g.sp_rows);
-            ++g.launches;
-        }
-        gp->slot[i] = slot;
+        sb.slot[i] = first + (int64_t)i * g.slot_cap;
+        sb.row_idx[i] = d.row_idx;
+        sb.n_rows[i] = (d.row_idx && d.n_rows > 0) ? d.n_rows : 0;
+        most = std::max(most, sb.n_rows[i]);
+        gp->slot[i] = sb.slot[i];
         gp->row_vals[i] = d.row_vals;
         gp->dense[i] = d.dense;
+    }
+    if (most > 0) {
+        scatter_slots_kernel<<<dim3((most + 255) / 256, nw), 256, 0, g.main>>>(sb, g.sp_rows);
+        ++g.launches;
     }
     return HPSGD_OK;
 }
@@ -1099,8 +1106,13 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
 
     // the map keeps the previous call's contents: every row starts again at "no slot" (-1)
     CUDA_TRY(cudaMemsetAsync(d->slot, 0xFF, (size_t)rows * 4, s));
-    if (have_rows)
-        scatter_slots_kernel<<<(desc->n_rows + 255) / 256, 256, 0, s>>>(d->slot, desc->row_idx, desc->n_rows, rows);
+    if (have_rows) {
+        SlotBatch sb{};
+        sb.slot[0] = d->slot;
+        sb.row_idx[0] = desc->row_idx;
+        sb.n_rows[0] = desc->n_rows;
+        scatter_slots_kernel<<<dim3((desc->n_rows + 255) / 256, 1), 256, 0, s>>>(sb, rows);
+    }
     BatchPtrs gp{};
     gp.dense[0] = desc->dense;
     gp.row_vals[0] = desc->row_vals;

@@ -54,22 +54,63 @@ __device__ __forceinline__ f8 zero8()
     return x;
 }
 
-// Eight consecutive gradient values of group o (o counts groups of 8 elements).
-// bf16 storage: one 128-bit load, each value widened exactly (bits << 16).
+// Eight consecutive gradient values of group o (o counts groups of 8 elements), as stored:
+// 32 bytes of fp32 or 16 bytes of bf16.  Loading and widening are separate steps so that a
+// thread can request several groups before it touches the first one.
+template <bool BF16>
+struct GradRaw;
+template <>
+struct GradRaw<false> {
+    f8 x;
+};
+template <>
+struct GradRaw<true> {
+    uint4 u;
+};
+
+template <bool BF16>
+__device__ __forceinline__ GradRaw<BF16> load_grad_raw(const void* g, int64_t o)
+{
+    GradRaw<BF16> raw;
+    if constexpr (BF16) {
+        asm volatile("ld.global.v4.b32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(raw.u.x), "=r"(raw.u.y), "=r"(raw.u.z), "=r"(raw.u.w)
+                     : "l"(reinterpret_cast<const uint4*>(g) + o));
+    } else {
+        raw.x = ld8(reinterpret_cast<const float*>(g) + o * 8);
+    }
+    return raw;
+}
+
+template <bool BF16>
+__device__ __forceinline__ GradRaw<BF16> zero_grad_raw()
+{
+    GradRaw<BF16> raw;
+    if constexpr (BF16) raw.u = make_uint4(0u, 0u, 0u, 0u);
+    else raw.x = zero8();
+    return raw;
+}
+
+// bf16 -> fp32 is exact: the 16 stored bits become the upper half of the binary32 pattern.
+template <bool BF16>
+__device__ __forceinline__ f8 widen_grad(const GradRaw<BF16>& raw)
+{
+    if constexpr (BF16) {
+        f8 x;
+        x.v[0] = __uint_as_float(raw.u.x << 16); x.v[1] = __uint_as_float(raw.u.x & 0xFFFF0000u);
+        x.v[2] = __uint_as_float(raw.u.y << 16); x.v[3] = __uint_as_float(raw.u.y & 0xFFFF0000u);
+        x.v[4] = __uint_as_float(raw.u.z << 16); x.v[5] = __uint_as_float(raw.u.z & 0xFFFF0000u);
+        x.v[6] = __uint_as_float(raw.u.w << 16); x.v[7] = __uint_as_float(raw.u.w & 0xFFFF0000u);
+        return x;
+    } else {
+        return raw.x;
+    }
+}
+
 template <bool BF16>
 __device__ __forceinline__ f8 load_grad8(const void* g, int64_t o)
 {
-    if constexpr (BF16) {
-        const uint4 u = __ldcs(reinterpret_cast<const uint4*>(g) + o);
-        f8 x;
-        x.v[0] = __uint_as_float(u.x << 16); x.v[1] = __uint_as_float(u.x & 0xFFFF0000u);
-        x.v[2] = __uint_as_float(u.y << 16); x.v[3] = __uint_as_float(u.y & 0xFFFF0000u);
-        x.v[4] = __uint_as_float(u.z << 16); x.v[5] = __uint_as_float(u.z & 0xFFFF0000u);
-        x.v[6] = __uint_as_float(u.w << 16); x.v[7] = __uint_as_float(u.w & 0xFFFF0000u);
-        return x;
-    } else {
-        return ld8(reinterpret_cast<const float*>(g) + o * 8);
-    }
+    return widen_grad<BF16>(load_grad_raw<BF16>(g, o));
 }
 
 // ---------------------------------------------------------------------------- local step
@@ -150,14 +191,21 @@ local_step_kernel(float* __restrict__ r_base, float* __restrict__ m_base, int64_
     }
 }
 
-// Row -> slot map of the sparse-row tensor: slot[row_idx[k]] = k (map pre-filled with -1).
-__global__ void scatter_slots_kernel(int32_t* __restrict__ slot, const int32_t* __restrict__ row_idx,
-                                     int32_t n_rows, int64_t rows)
+// Row -> slot maps of the sparse-row tensor: slot_i[row_idx_i[k]] = k for every worker i of
+// a batch (blockIdx.y), the maps pre-filled with -1.
+struct SlotBatch {
+    int32_t* slot[kMaxBatch];
+    const int32_t* row_idx[kMaxBatch];
+    int32_t n_rows[kMaxBatch];
+};
+
+__global__ void scatter_slots_kernel(SlotBatch sb, int64_t rows)
 {
+    const int i = blockIdx.y;
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k < n_rows) {
-        const int32_t row = row_idx[k];
-        if (row >= 0 && row < rows) slot[row] = k;
+    if (k < sb.n_rows[i]) {
+        const int32_t row = sb.row_idx[i][k];
+        if (row >= 0 && row < rows) sb.slot[i][row] = k;
     }
 }
 
@@ -239,19 +287,36 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
 // same order, same results as merge_kernel followed by local_step_kernel, but per index
 // it moves (K r + w + D) in, (w + D) out, then per worker (g + m) in, (r + m) out:
 // (5K + 4) * 4 bytes with fp32 gradients instead of (7K + 4) * 4.
-template <bool BF16, bool SPARSE>
-__device__ __forceinline__ f8 fused_grad8(const BatchPtrs& gp, const SparseSeg& seg, int i, int64_t o)
+// Position of a group inside the sparse-row tensor.
+struct SegPos {
+    bool inside;
+    int64_t row;
+    int64_t col8;
+};
+
+__device__ __forceinline__ SegPos seg_pos(const SparseSeg& seg, int64_t o)
 {
-    if (SPARSE) {
-        if (o >= seg.o_begin && o < seg.o_end) {
-            const int64_t rel = o - seg.o_begin;
-            const int64_t row = rel / seg.cols8;
-            const int32_t s = __ldg(gp.slot[i] + row);
-            if (s < 0) return zero8();
-            return load_grad8<BF16>(gp.row_vals[i], (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
-        }
+    SegPos sp{false, 0, 0};
+    if (o >= seg.o_begin && o < seg.o_end) {
+        const int64_t rel = o - seg.o_begin;
+        sp.inside = true;
+        sp.row = rel / seg.cols8;
+        sp.col8 = rel - sp.row * seg.cols8;
     }
-    return load_grad8<BF16>(gp.dense[i], o);
+    return sp;
+}
+
+// Stored gradient group of worker i: from its dense buffer, or, inside the sparse-row tensor,
+// from slot `s` of its row values (s < 0: the row has no gradient).
+template <bool BF16, bool SPARSE>
+__device__ __forceinline__ GradRaw<BF16> fused_grad_raw(const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp,
+                                                        int32_t s, int i, int64_t o)
+{
+    if (SPARSE && sp.inside) {
+        if (s < 0) return zero_grad_raw<BF16>();
+        return load_grad_raw<BF16>(gp.row_vals[i], (int64_t)s * seg.cols8 + sp.col8);
+    }
+    return load_grad_raw<BF16>(gp.dense[i], o);
 }
 
 template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
@@ -266,6 +331,17 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
         const int64_t e = o * 8;
+        // every worker's row -> slot entry is requested up front, so that the gradient loads
+        // of the step phase do not wait on a dependent lookup
+        SegPos sp{false, 0, 0};
+        int32_t sl[KT > 0 ? KT : 1];
+        if (SPARSE) {
+            sp = seg_pos(seg, o);
+            if (KT > 0 && sp.inside) {
+#pragma unroll
+                for (int i = 0; i < (KT > 0 ? KT : 1); ++i) sl[i] = __ldg(gp.slot[i] + sp.row);
+            }
+        }
         // ---- merge
         const f8 wv = ld8(w + e);
         f8 dv = zero8();
@@ -317,25 +393,35 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
         int i0 = 0;
 #pragma unroll
         for (; i0 + B <= Kn; i0 += B) {
-            f8 gg[B], mm[B];
+            GradRaw<BF16> graw[B];
+            f8 mm[B];
+            int32_t sb[B];
+            if (SPARSE && sp.inside) {
+#pragma unroll
+                for (int b = 0; b < B; ++b) sb[b] = KT > 0 ? sl[i0 + b] : __ldg(gp.slot[i0 + b] + sp.row);
+            }
 #pragma unroll
             for (int b = 0; b < B; ++b) {
-                gg[b] = fused_grad8<BF16, SPARSE>(gp, seg, i0 + b, o);
+                graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, sb[b], i0 + b, o);
                 if (MOM) mm[b] = ld8(m + (int64_t)(i0 + b) * stride + e);
             }
 #pragma unroll
             for (int b = 0; b < B; ++b) {
+                const f8 gg = widen_grad<BF16>(graw[b]);
                 f8 rr;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) rr.v[q] = step1<MOM, WD>(gg[b].v[q], mm[b].v[q], wn.v[q], p);
+                for (int q = 0; q < 8; ++q) rr.v[q] = step1<MOM, WD>(gg.v[q], mm[b].v[q], wn.v[q], p);
                 st8(r + (int64_t)(i0 + b) * stride + e, rr);
                 if (MOM) st8(m + (int64_t)(i0 + b) * stride + e, mm[b]);
             }
         }
         for (; i0 < Kn; ++i0) {
-            f8 gg = fused_grad8<BF16, SPARSE>(gp, seg, i0, o);
+            int32_t s1 = -1;
+            if (SPARSE && sp.inside) s1 = __ldg(gp.slot[i0] + sp.row);
+            const GradRaw<BF16> graw = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, s1, i0, o);
             f8 mm;
             if (MOM) mm = ld8(m + (int64_t)i0 * stride + e);
+            const f8 gg = widen_grad<BF16>(graw);
             f8 rr;
 #pragma unroll
             for (int q = 0; q < 8; ++q) rr.v[q] = step1<MOM, WD>(gg.v[q], mm.v[q], wn.v[q], p);
