@@ -64,7 +64,14 @@ def fused_bytes_per_index(cfg):
 # DRAM bytes per parameter index (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
 # capture divided by the indices of that launch), keyed by (kernel, K, gradient dtype), with
 # the SHA-1 of the kernel source the capture was taken from.  A changed source voids them.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200105 GB read + 2.123378 GB written over 16,000,000 indices
+    ("merge_step_kernel", 16, "f32"): {"bytes_per_index": 5.323483e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
+    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152239 GB + 1.093508 GB
+    ("merge_kernel", 16, "f32"): {"bytes_per_index": 2.245747e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
+    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072009 GB + 1.993030 GB (all 16 workers in one launch)
+    ("local_step_kernel", 16, "f32"): {"bytes_per_index": 5.065039e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
+}
 
 
 def ncu_traffic(kernel, cfg, algorithmic_bytes_per_launch):
@@ -199,6 +206,29 @@ def run_reference(args, cfg):
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
+
+
+def cut_workload(cfg, max_params):
+    """The same rule, K and gradients on the leading part of the parameter set: tensors are taken
+    in order until `max_params` is reached, the one that crosses it is shortened (a sparse-row
+    tensor keeps whole rows).  Used for profiler captures, which must stay small."""
+    sizes, total, sparse = [], 0, None
+    for t, size in enumerate(cfg.sizes):
+        room = max_params - total
+        if room < 64:
+            break
+        if cfg.sparse and t == cfg.sparse[0]:
+            cols = cfg.sparse[2]
+            rows = max(1, min(cfg.sparse[1], room // cols))
+            size = rows * cols
+            sparse = (len(sizes), rows, cols)
+        else:
+            size = min(size, room)
+        sizes.append(size)
+        total += size
+    cut = cfg.subset(cfg.name, sizes, sparse=sparse)
+    object.__setattr__(cut, "note", "%s, cut to its first %d parameters" % (cfg.note, total))
+    return cut
 
 
 def workload_config(cfg, extra=None):
@@ -472,10 +502,14 @@ def main():
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--e2e-host-buffers", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU oracle baseline budget (0 = skip)")
+    ap.add_argument("--max-params", type=int, default=0,
+                    help="cut the workload to its first N parameters (for small profiler captures)")
     ap.add_argument("--ref-sample", type=int, default=4_000_000, help="parameters per step of --impl reference")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
     cfg = workloads.get(args.workload)
+    if args.max_params:
+        cfg = cut_workload(cfg, args.max_params)
 
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
