@@ -42,6 +42,11 @@
  *   - staleness = 0 is a test mode that commits the fresh average at once (Eq. 2:
  *     the global model becomes the mean of the replicas, i.e. Local SGD, Algorithm 1).
  *
+ * A second, independent set of functions (ref_acc_*) follows Algorithms 2 and 3 in the
+ * form they are printed, for the paper's plain SGD: explicit accumulated gradients per
+ * worker, AllReduce of those accumulators (mean), and the delayed commit
+ * w <- w - mu * (mean gradients all-reduced at the previous synchronisation).
+ *
  * Pins (tests/, run without a GPU): hand-worked K=2, P=4 examples; the closed form of
  * Eq. 1 in binary64; a separate literal transcription of Algorithms 2 and 3 with explicit
  * gradient accumulators; K=1 against a library SGD/momentum optimiser; Local SGD model
@@ -110,9 +115,95 @@ void sync_merge(RefState* s)
     s->merges += 1;
 }
 
+/* ---- Algorithms 2 and 3 as printed: gradient-accumulation form, plain SGD ---- */
+struct AccState {
+    int64_t P = 0;
+    int K = 0;
+    float mu = 0.f;
+    bool synced_valid = false;           // an AllReduce result from the previous synchronisation exists
+    int64_t syncs = 0;
+    std::vector<float> w;                // global model
+    std::vector<float> synced;           // result of the last AllReduce (mean accumulated gradient)
+    std::vector<std::vector<float>> r;   // replicas
+    std::vector<std::vector<float>> a;   // accumulated gradients
+};
+
+/* Algorithm 2: "update replica" r_i = r_i - mu*g and "accumulate gradients" a_i = a_i + g. */
+void acc_local_step(AccState* s, int i, const float* g)
+{
+    float* r = s->r[i].data();
+    float* a = s->a[i].data();
+    for (int64_t j = 0; j < s->P; ++j) {
+        r[j] = std::fmaf(-s->mu, g[j], r[j]);
+        a[j] = a[j] + g[j];
+    }
+}
+
+/* Algorithm 3: commit the previous AllReduce result, AllReduce the accumulators (mean over
+ * the K workers, left to right), reset them, and re-clone the replicas (Algorithm 2). */
+void acc_sync(AccState* s)
+{
+    const float fK = static_cast<float>(s->K);
+    for (int64_t j = 0; j < s->P; ++j) {
+        if (s->synced_valid) s->w[j] = std::fmaf(-s->mu, s->synced[j], s->w[j]);
+        float sum = s->a[0][j];
+        for (int i = 1; i < s->K; ++i) sum = sum + s->a[i][j];
+        s->synced[j] = sum / fK;
+        for (int i = 0; i < s->K; ++i) {
+            s->a[i][j] = 0.f;
+            s->r[i][j] = s->w[j];
+        }
+    }
+    s->synced_valid = true;
+    s->syncs += 1;
+}
+
 }  // namespace
 
 extern "C" {
+
+void* ref_acc_create(int64_t P, int K, float lr)
+{
+    if (P <= 0 || K <= 0) return nullptr;
+    AccState* s = new (std::nothrow) AccState;
+    if (!s) return nullptr;
+    s->P = P; s->K = K; s->mu = lr;
+    s->w.assign(P, 0.f);
+    s->synced.assign(P, 0.f);
+    s->r.assign(K, std::vector<float>(P, 0.f));
+    s->a.assign(K, std::vector<float>(P, 0.f));
+    return s;
+}
+
+void ref_acc_destroy(void* h) { delete static_cast<AccState*>(h); }
+
+void ref_acc_set_global(void* h, const float* w0)
+{
+    AccState* s = static_cast<AccState*>(h);
+    s->w.assign(w0, w0 + s->P);
+    std::fill(s->synced.begin(), s->synced.end(), 0.f);
+    s->synced_valid = false;
+    s->syncs = 0;
+    for (int i = 0; i < s->K; ++i) {
+        s->r[i] = s->w;
+        std::fill(s->a[i].begin(), s->a[i].end(), 0.f);
+    }
+}
+
+int ref_acc_local_step(void* h, int worker, const float* g)
+{
+    AccState* s = static_cast<AccState*>(h);
+    if (worker < 0 || worker >= s->K) return -1;
+    acc_local_step(s, worker, g);
+    return 0;
+}
+
+void ref_acc_sync(void* h) { acc_sync(static_cast<AccState*>(h)); }
+
+const float* ref_acc_get_global(void* h) { return static_cast<AccState*>(h)->w.data(); }
+const float* ref_acc_get_synced(void* h) { return static_cast<AccState*>(h)->synced.data(); }
+const float* ref_acc_get_replica(void* h, int i) { return static_cast<AccState*>(h)->r[i].data(); }
+const float* ref_acc_get_accumulated(void* h, int i) { return static_cast<AccState*>(h)->a[i].data(); }
 
 void* ref_create(int64_t P, int K, float lr, float momentum, float weight_decay, int staleness)
 {

@@ -56,6 +56,22 @@ def _bind(lib):
         getattr(lib, name).argtypes = [vp, ci]
     lib.ref_merges.restype = i64
     lib.ref_merges.argtypes = [vp]
+    lib.ref_acc_create.restype = vp
+    lib.ref_acc_create.argtypes = [i64, ci, f32]
+    lib.ref_acc_destroy.restype = None
+    lib.ref_acc_destroy.argtypes = [vp]
+    lib.ref_acc_set_global.restype = None
+    lib.ref_acc_set_global.argtypes = [vp, vp]
+    lib.ref_acc_local_step.restype = ci
+    lib.ref_acc_local_step.argtypes = [vp, ci, vp]
+    lib.ref_acc_sync.restype = None
+    lib.ref_acc_sync.argtypes = [vp]
+    for name in ("ref_acc_get_global", "ref_acc_get_synced"):
+        getattr(lib, name).restype = ctypes.POINTER(ctypes.c_float)
+        getattr(lib, name).argtypes = [vp]
+    for name in ("ref_acc_get_replica", "ref_acc_get_accumulated"):
+        getattr(lib, name).restype = ctypes.POINTER(ctypes.c_float)
+        getattr(lib, name).argtypes = [vp, ci]
     return lib
 
 
@@ -137,3 +153,51 @@ class RefHPSGD:
     @property
     def merges(self):
         return int(self._lib.ref_merges(self._h))
+
+
+class RefHPSGDAccum:
+    """Algorithms 2 and 3 as printed (plain SGD): explicit accumulated gradients per worker."""
+
+    def __init__(self, P, K, lr, lib=None):
+        self._lib = lib or load()
+        self.P, self.K = int(P), int(K)
+        self._h = self._lib.ref_acc_create(self.P, self.K, lr)
+        if not self._h:
+            raise ValueError("ref_acc_create rejected the arguments")
+
+    def close(self):
+        if self._h:
+            self._lib.ref_acc_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def set_global(self, w0):
+        a = np.ascontiguousarray(w0, dtype=np.float32)
+        assert a.size == self.P
+        self._lib.ref_acc_set_global(self._h, a.ctypes.data)
+
+    def local_step(self, worker, g):
+        a = np.ascontiguousarray(g, dtype=np.float32)
+        assert a.size == self.P
+        if self._lib.ref_acc_local_step(self._h, worker, a.ctypes.data):
+            raise ValueError("bad worker index")
+
+    def sync_merge(self):
+        self._lib.ref_acc_sync(self._h)
+
+    def _view(self, ptr):
+        return np.ctypeslib.as_array(ptr, shape=(self.P,)).copy()
+
+    def get_global(self):
+        return self._view(self._lib.ref_acc_get_global(self._h))
+
+    def get_synced(self):
+        return self._view(self._lib.ref_acc_get_synced(self._h))
+
+    def get_replica(self, i):
+        return self._view(self._lib.ref_acc_get_replica(self._h, i))
+
+    def get_accumulated(self, i):
+        return self._view(self._lib.ref_acc_get_accumulated(self._h, i))

@@ -10,7 +10,7 @@ import os
 
 import numpy as np
 
-from oracle.ref import RefHPSGD
+from oracle.ref import RefHPSGD, RefHPSGDAccum
 
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
@@ -377,6 +377,73 @@ def pin_storage_variants(lib):
         b.close()
 
 
+# ------------------------------------------------------------------ gradient-accumulation form
+def pin_accum_worked_example(lib):
+    """The printed form on the hand-worked plain-SGD rounds: same replicas and global model;
+    the AllReduce result is the mean gradient, i.e. -D/mu of the replica-change form."""
+    mu, w0, grads, cases = parse_worked(os.path.join(GOLDEN, "worked_k2_p4.txt"))
+    c = [c for c in cases if c["beta"] == 0 and c["lambda"] == 0 and c["staleness"] == 1][0]
+    o = RefHPSGDAccum(4, 2, mu, lib=lib)
+    o.set_global(w0)
+    for t in range(3):
+        for i in range(2):
+            o.local_step(i, np.array(grads[(t, i)], dtype=np.float32))
+            np.testing.assert_array_equal(o.get_replica(i), np.float32(c["r"][(t, i)]))
+        acc = [o.get_accumulated(i) for i in range(2)]
+        np.testing.assert_array_equal(acc[0], np.float32(grads[(t, 0)]))
+        o.sync_merge()
+        np.testing.assert_array_equal(o.get_global(), np.float32(c["w"][t]))
+        np.testing.assert_array_equal(o.get_synced(), -np.float32(c["D"][t]) / np.float32(mu))
+        for i in range(2):
+            np.testing.assert_array_equal(o.get_replica(i), o.get_global())
+            np.testing.assert_array_equal(o.get_accumulated(i), 0)
+    o.close()
+
+
+def pin_accum_literal_and_closed_form(lib):
+    """The printed form against its binary64 transcription with status/counter flags, the
+    closed form of Eq. 1, and the replica-change oracle (Eq. 1 == Eq. 2)."""
+    rng = _rng(41)
+    for trial in range(8):
+        K = int(rng.integers(1, 6))
+        P = int(rng.integers(1, 9))
+        busy = int(rng.integers(0, 4))
+        syncs = int(rng.integers(2, 6))
+        epochs = 1 + (syncs - 1) * (busy + 1)
+        mu = float(rng.choice([0.5, 0.1, 0.03]))
+        w0 = rng.uniform(-1, 1, P).astype(np.float32)
+        grads = rng.uniform(-1, 1, (epochs, K, P)).astype(np.float32)
+        want_w, _ = literal_hpsgd(w0, grads.astype(np.float64), mu, busy)
+        acc = RefHPSGDAccum(P, K, mu, lib=lib)
+        rep = RefHPSGD(P, K, mu, 0.0, 0.0, 1, lib=lib)
+        acc.set_global(w0)
+        rep.set_global(w0)
+        e = 0
+        committed = np.zeros(P)
+        period_sum = None
+        for s in range(syncs):
+            steps = 1 if s == 0 else busy + 1
+            this_period = np.zeros(P)
+            for _ in range(steps):
+                for i in range(K):
+                    acc.local_step(i, grads[e, i])
+                    rep.local_step(i, grads[e, i])
+                this_period += grads[e].astype(np.float64).sum(axis=0)
+                e += 1
+            if period_sum is not None:
+                committed += period_sum                 # the previous period lands now
+            period_sum = this_period
+            acc.sync_merge()
+            rep.sync_merge()
+            np.testing.assert_allclose(acc.get_global(), want_w[s], rtol=0, atol=4e-6)
+            closed = w0.astype(np.float64) - np.float64(np.float32(mu)) / K * committed
+            np.testing.assert_allclose(acc.get_global(), closed, rtol=0, atol=4e-6)
+            np.testing.assert_allclose(acc.get_global(), rep.get_global(), rtol=0, atol=4e-6)
+            np.testing.assert_allclose(acc.get_synced(), this_period / K, rtol=1e-5, atol=1e-7)
+        acc.close()
+        rep.close()
+
+
 ALL_PINS = [
     pin_worked_examples,
     pin_literal_algorithms,
@@ -388,4 +455,6 @@ ALL_PINS = [
     pin_equal_gradients,
     pin_staleness_is_one_sync_shift,
     pin_storage_variants,
+    pin_accum_worked_example,
+    pin_accum_literal_and_closed_form,
 ]

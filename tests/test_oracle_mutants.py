@@ -24,6 +24,14 @@ MUTANTS = {
     "clone_before_commit": [("float Dnew = acc / fK;",
                              "float Dnew = acc / fK; for (int i = 0; i < s->K; ++i) s->r[i][j] = s->w[j];"),
                             ("        for (int i = 0; i < s->K; ++i) s->r[i][j] = s->w[j];\n", "")],
+    "accum_not_reset": ("s->a[i][j] = 0.f;", ""),
+    "accum_sum_not_mean": ("s->synced[j] = sum / fK;", "s->synced[j] = sum;"),
+    "accum_commit_without_lr": ("s->w[j] = std::fmaf(-s->mu, s->synced[j], s->w[j]);", "s->w[j] = s->w[j] - s->synced[j];"),
+    "accum_commit_not_delayed": ("if (s->synced_valid) s->w[j] = std::fmaf(-s->mu, s->synced[j], s->w[j]);",
+                                 "s->w[j] = std::fmaf(-s->mu, s->a[0][j], s->w[j]);"),
+    "accum_replica_not_updated": ("r[j] = std::fmaf(-s->mu, g[j], r[j]);\n        a[j]", "a[j]"),
+    "accum_first_worker_twice": ("for (int i = 1; i < s->K; ++i) sum = sum + s->a[i][j];",
+                                 "for (int i = 1; i < s->K; ++i) sum = sum + s->a[0][j];"),
     "pending_overwritten_early": ("float Dnew = acc / fK;", "float Dnew = acc / fK; s->D[j] = Dnew;"),
 }
 
