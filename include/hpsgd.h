@@ -141,6 +141,21 @@ const float* hpsgd_get_global(void);
  */
 int64_t hpsgd_layout_padded(int n_tensors, const int64_t* sizes, int64_t* offsets_out);
 
+/*
+ * What each worker carries between synchronisations, for the next hpsgd_init:
+ *   HPSGD_FORM_REPLICA_CHANGE (default): only the replica; its displacement from w stands
+ *     for the accumulated gradient (Eq. 2), and the merge averages replica changes.
+ *   HPSGD_FORM_GRADIENT_ACCUMULATION: Algorithms 2 and 3 as printed, for the paper's plain
+ *     SGD (momentum must be 0, no weight decay).  Local step: r_i = r_i - mu*g (one FMA) and
+ *     a_i = a_i + g.  Merge: w = w - mu*ghat (one FMA) if a previous AllReduce result ghat
+ *     exists (staleness 0: the fresh mean instead); ghat = (a_0 + ... + a_{K-1}) / K left to
+ *     right; a_i = 0; r_i = w.  In this form hpsgd_get_pending returns ghat, the second
+ *     pointer of hpsgd_get_replica returns a_i, HPSGD_ARENA_MOMENTUM must be set when sizing
+ *     an arena, and HPSGD_OPT_FUSE has no effect.
+ */
+enum { HPSGD_FORM_REPLICA_CHANGE = 0, HPSGD_FORM_GRADIENT_ACCUMULATION = 1 };
+int hpsgd_set_form(int form);
+
 /* Declare the tensor sizes (host array, each > 0) used by the next hpsgd_init. */
 int hpsgd_set_layout(int n_tensors, const int64_t* sizes);
 

@@ -19,6 +19,7 @@ HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP = 0, 1, 2
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
+HPSGD_FORM_REPLICA_CHANGE, HPSGD_FORM_GRADIENT_ACCUMULATION = 0, 1
 HPSGD_NOALLOC_MAX_ROWS = 262144
 
 
@@ -45,6 +46,7 @@ SIGNATURES = {
     "hpsgd_get_global": (_vp, []),
     "hpsgd_layout_padded": (_i64, [_ci, _P(_i64), _P(_i64)]),
     "hpsgd_set_layout": (_ci, [_ci, _P(_i64)]),
+    "hpsgd_set_form": (_ci, [_ci]),
     "hpsgd_arena_bytes": (_sz, [_i64, _ci, _ci, _i64]),
     "hpsgd_bind": (_ci, [_vp, _sz, _vp, _vp]),
     "hpsgd_set_option": (_ci, [_ci, _f64]),
@@ -153,6 +155,10 @@ def hpsgd_layout_padded(sizes):
 def hpsgd_set_layout(sizes):
     n = len(sizes)
     return _check(load().hpsgd_set_layout(n, (_i64 * n)(*[int(s) for s in sizes])))
+
+
+def hpsgd_set_form(form):
+    return _check(load().hpsgd_set_form(int(form)))
 
 
 def hpsgd_arena_bytes(P_pad, K, flags=0, sparse_rows=0):

@@ -59,6 +59,7 @@ struct Pending {                // configuration collected before hpsgd_init
     size_t arena_bytes = 0;
     cudaStream_t main = nullptr, side = nullptr;
     bool have_streams = false;
+    int form = HPSGD_FORM_REPLICA_CHANGE;
 } g_pending;
 
 struct Ctx {
@@ -83,6 +84,7 @@ struct Ctx {
     std::vector<char> local_recorded, merge_unwaited;
     bool D_valid = false;
     int64_t merges = 0;
+    int form = HPSGD_FORM_REPLICA_CHANGE;  // what the workers carry: replica change or accumulated gradients
     int fuse = 0;                          // carry a merge into the next batched local step
     bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
     int deferred_flags = 0;
@@ -232,6 +234,20 @@ void launch_local_d(bool mom, bool wd, bool sparse, const LocalLaunch& L)
     else launch_local_s<BF16, false, false>(sparse, L);
 }
 
+// Gradient-accumulation form: r -= mu*g, a += g (the accumulators live where momentum would).
+void launch_accum_step(bool sparse, const LocalLaunch& L)
+{
+    dim3 grid(hot_grid(L.n), L.nw);
+    const bool bf = g.grad_dtype == HPSGD_BF16;
+#define HPSGD_ACCUM_CASE(B, S) \
+    accum_step_kernel<B, S><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.o0, L.n, L.p.neg_mu)
+    if (bf && sparse) HPSGD_ACCUM_CASE(true, true);
+    else if (bf) HPSGD_ACCUM_CASE(true, false);
+    else if (sparse) HPSGD_ACCUM_CASE(false, true);
+    else HPSGD_ACCUM_CASE(false, false);
+#undef HPSGD_ACCUM_CASE
+}
+
 // Enqueue the local step of workers [w0, w0 + nw) on the main stream, chunk by chunk.
 int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
 {
@@ -256,7 +272,8 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
         L.o0 = lo; L.n = hi - lo;
         EventPair ep{};
         TRY(prof_begin(g.main, HPSGD_KERNEL_LOCAL_STEP, &ep));
-        if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
+        if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) launch_accum_step(sparse, L);
+        else if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
         else launch_local_d<false>(mom, wd, sparse, L);
         ++g.launches;
         TRY(prof_end(g.main, &ep));
@@ -419,6 +436,12 @@ void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
     merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags);
 }
 
+template <int KT>
+void launch_accum_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
+{
+    accum_merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.m, g.stride, g.K, o0, n, flags, -g.lr);
+}
+
 // Enqueue one merge, chunk by chunk, on the side stream (main stream without overlap).
 int enqueue_merge(int flags)
 {
@@ -433,11 +456,20 @@ int enqueue_merge(int flags)
         }
         EventPair ep{};
         TRY(prof_begin(s, HPSGD_KERNEL_MERGE, &ep));
-        switch (g.K) {
-        case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
-        case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
-        case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
-        default: launch_merge<0>(s, lo, hi - lo, flags); break;
+        if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) {
+            switch (g.K) {
+            case 4: launch_accum_merge<4>(s, lo, hi - lo, flags); break;
+            case 8: launch_accum_merge<8>(s, lo, hi - lo, flags); break;
+            case 16: launch_accum_merge<16>(s, lo, hi - lo, flags); break;
+            default: launch_accum_merge<0>(s, lo, hi - lo, flags); break;
+            }
+        } else {
+            switch (g.K) {
+            case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
+            case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
+            case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
+            default: launch_merge<0>(s, lo, hi - lo, flags); break;
+            }
         }
         ++g.launches;
         TRY(prof_end(s, &ep));
@@ -555,6 +587,15 @@ int64_t hpsgd_layout_padded(int n_tensors, const int64_t* sizes, int64_t* offset
     return pad;
 }
 
+int hpsgd_set_form(int form)
+{
+    if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_set_form must precede hpsgd_init");
+    if (form != HPSGD_FORM_REPLICA_CHANGE && form != HPSGD_FORM_GRADIENT_ACCUMULATION)
+        return fail(HPSGD_E_BADARG, "unknown form %d", form);
+    g_pending.form = form;
+    return HPSGD_OK;
+}
+
 int hpsgd_set_layout(int n_tensors, const int64_t* sizes)
 {
     if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_set_layout must precede hpsgd_init");
@@ -599,6 +640,8 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     if (K <= 0 || K > 256) return fail(HPSGD_E_BADARG, "K must be in [1, 256]");
     if (!(lr >= 0.f)) return fail(HPSGD_E_BADARG, "lr must be >= 0");
     if (!(momentum >= 0.f && momentum < 1.f)) return fail(HPSGD_E_BADARG, "momentum must be in [0, 1)");
+    if (g_pending.form == HPSGD_FORM_GRADIENT_ACCUMULATION && momentum != 0.f)
+        return fail(HPSGD_E_BADARG, "the gradient-accumulation form is the paper's plain SGD: momentum must be 0");
     std::vector<int64_t> sizes = g_pending.sizes;
     if (sizes.empty()) sizes.push_back(P);
     int64_t sum = 0;
@@ -620,7 +663,8 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.sizes = sizes;
     g.P_pad = layout_of(sizes, &g.offsets, &g.starts);
     g.stride = (g.P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
-    const bool mom = momentum != 0.f;
+    g.form = g_pending.form;
+    const bool mom = momentum != 0.f || g.form == HPSGD_FORM_GRADIENT_ACCUMULATION;   // K extra rows: m_i or a_i
     const ArenaPlan a = plan_arena(g.stride, K, mom);
 
     if (g_pending.arena) {
@@ -712,6 +756,8 @@ int hpsgd_set_option(int key, double value)
     switch (key) {
     case HPSGD_OPT_WEIGHT_DECAY:
         if (!(value >= 0.0)) return fail(HPSGD_E_BADARG, "weight decay must be >= 0");
+        if (value != 0.0 && g.form == HPSGD_FORM_GRADIENT_ACCUMULATION)
+            return fail(HPSGD_E_BADARG, "the gradient-accumulation form has no weight decay");
         g.lambda = (float)value;
         return HPSGD_OK;
     case HPSGD_OPT_STALENESS:
@@ -890,7 +936,7 @@ int hpsgd_sync_merge(void)
     else if (g.D_valid) flags |= kMergeApplyPending;
     g.D_valid = true;
     g.merges += 1;
-    if (g.fuse) {
+    if (g.fuse && g.form == HPSGD_FORM_REPLICA_CHANGE) {
         g.merge_deferred = true;
         g.deferred_flags = flags;
         return HPSGD_OK;

@@ -280,6 +280,108 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
     }
 }
 
+// ---------------------------------------------------------------------------- gradient-accumulation form
+// Algorithms 2 and 3 as printed, plain SGD: each worker keeps its accumulated gradients a_i.
+//   local step:  r_i = r_i - mu*g (one FMA) ; a_i = a_i + g
+//   merge:       w = w - mu*ghat (one FMA, if a previous AllReduce result ghat exists; with
+//                staleness 0 the fresh mean is committed instead) ;
+//                ghat = (a_0 + ... + a_{K-1}) / K left to right ; a_i = 0 ; r_i = w
+template <bool BF16, bool SPARSE>
+__global__ void __launch_bounds__(kHotThreads)
+accum_step_kernel(float* __restrict__ r_base, float* __restrict__ a_base, int64_t stride,
+                  int w0, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, float neg_mu)
+{
+    const int wk = blockIdx.y;
+    float* __restrict__ r = r_base + (int64_t)(w0 + wk) * stride;
+    float* __restrict__ a = a_base + (int64_t)(w0 + wk) * stride;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        f8 rr = ld8(r + o * 8);
+        f8 aa = ld8(a + o * 8);
+        GradRaw<BF16> raw;
+        bool dense_src = true;
+        if (SPARSE) {
+            if (o >= seg.o_begin && o < seg.o_end) {
+                dense_src = false;
+                const int64_t rel = o - seg.o_begin;
+                const int64_t row = rel / seg.cols8;
+                const int32_t s = __ldg(gp.slot[wk] + row);
+                if (s >= 0) raw = load_grad_raw<BF16>(gp.row_vals[wk], (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
+                else raw = zero_grad_raw<BF16>();
+            }
+        }
+        if (dense_src) raw = load_grad_raw<BF16>(gp.dense[wk], o);
+        const f8 gg = widen_grad<BF16>(raw);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            rr.v[q] = __fmaf_rn(neg_mu, gg.v[q], rr.v[q]);
+            aa.v[q] = __fadd_rn(aa.v[q], gg.v[q]);
+        }
+        st8(r + o * 8, rr);
+        st8(a + o * 8, aa);
+    }
+}
+
+template <int KT>
+__global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
+accum_merge_kernel(float* __restrict__ w, float* __restrict__ ghat, float* __restrict__ r, float* __restrict__ a,
+                   int64_t stride, int K, int64_t o0, int64_t n, int flags, float neg_mu)
+{
+    const int Kn = KT > 0 ? KT : K;
+    const float fK = (float)Kn;
+    const f8 zero = zero8();
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        const int64_t e = o * 8;
+        const f8 wv = ld8(w + e);
+        f8 gv = zero;
+        if (flags & kMergeApplyPending) gv = ld8(ghat + e);
+        f8 sum;
+        if constexpr (KT > 0) {
+            f8 av[KT];
+#pragma unroll
+            for (int i = 0; i < KT; ++i) av[i] = ld8(a + (int64_t)i * stride + e);
+            sum = av[0];
+#pragma unroll
+            for (int i = 1; i < KT; ++i)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) sum.v[q] = __fadd_rn(sum.v[q], av[i].v[q]);
+        } else {
+            sum = ld8(a + e);
+            int i = 1;
+            for (; i + 4 <= K; i += 4) {
+                f8 av[4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) av[b] = ld8(a + (int64_t)(i + b) * stride + e);
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) sum.v[q] = __fadd_rn(sum.v[q], av[b].v[q]);
+            }
+            for (; i < K; ++i) {
+                const f8 ai = ld8(a + (int64_t)i * stride + e);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) sum.v[q] = __fadd_rn(sum.v[q], ai.v[q]);
+            }
+        }
+        f8 gnew, wn;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            gnew.v[q] = __fdiv_rn(sum.v[q], fK);
+            wn.v[q] = wv.v[q];
+            if (flags & kMergeImmediate) wn.v[q] = __fmaf_rn(neg_mu, gnew.v[q], wv.v[q]);
+            else if (flags & kMergeApplyPending) wn.v[q] = __fmaf_rn(neg_mu, gv.v[q], wv.v[q]);
+        }
+        st8(w + e, wn);
+        st8(ghat + e, gnew);
+#pragma unroll 4
+        for (int i = 0; i < Kn; ++i) {
+            st8(a + (int64_t)i * stride + e, zero);
+            st8(r + (int64_t)i * stride + e, wn);
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------- merge + next local step
 // The merge followed by the first local step of every worker, in one pass: the clone
 // r_i = w never goes to memory, it is the starting point of r_i - mu*m_i directly

@@ -35,18 +35,19 @@ def to_device(a: np.ndarray) -> torch.Tensor:
 
 
 @contextlib.contextmanager
-def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, lend_arena=False, streams=False, canary=False):
+def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, lend_arena=False, streams=False, canary=False):
     """hpsgd_init for a workload (layout, options, optional lent arena/streams); destroys on exit."""
     hp.hpsgd_destroy()
     lay = cfg.layout
     keep = {}
     if len(cfg.sizes) > 1:
         hp.hpsgd_set_layout(list(cfg.sizes))
+    hp.hpsgd_set_form(form)
     if lend_arena or streams:
         arena, nbytes, main, side = None, 0, None, None
         if lend_arena:
             rows = cfg.sparse[1] if cfg.sparse else 0
-            nbytes = hp.hpsgd_arena_bytes(lay.P_pad, cfg.K, hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0, rows)
+            nbytes = hp.hpsgd_arena_bytes(lay.P_pad, cfg.K, hp.HPSGD_ARENA_MOMENTUM if (cfg.momentum or form) else 0, rows)
             guard = 4096 if canary else 0
             buf = torch.full((nbytes + 2 * guard + 256,), 0xA5, dtype=torch.uint8, device=DEV)
             base = buf.data_ptr() + guard
@@ -104,7 +105,7 @@ def gpu_state(cfg):
     for i in range(cfg.K):
         r, m = hp.hpsgd_get_replica(i)
         rs.append(gpu_flat(r, cfg))
-        ms.append(gpu_flat(m, cfg) if m else None)
+        ms.append(gpu_flat(m, cfg) if m else None)      # momentum, or accumulated gradients
     return w, D, rs, ms
 
 
@@ -252,3 +253,48 @@ def stratified_sample(cfg, n_random=1 << 18, edge=64, seed=12345) -> np.ndarray:
     rng = np.random.default_rng(seed)
     picks.append(rng.integers(0, cfg.P, size=n_random))
     return np.unique(np.concatenate(picks)).astype(np.int64)
+
+
+def run_both_accum(cfg, T, *, staleness=1, overlap=1, chunks=1, batched=False, steps_per_round=1, session_kw=None):
+    """Gradient-accumulation form (Algorithms 2/3 as printed) on the GPU and on the oracle."""
+    from oracle.ref import RefHPSGDAccum
+    assert staleness == 1 and not cfg.momentum and not cfg.weight_decay
+    o = RefHPSGDAccum(cfg.P, cfg.K, cfg.lr)
+    o.set_global(cfg.initial_global())
+    with session(cfg, staleness=staleness, overlap=overlap, chunks=chunks, form=hp.HPSGD_FORM_GRADIENT_ACCUMULATION,
+                 **(session_kw or {})):
+        step = 0
+        for t in range(T):
+            keep = []
+            for h in range(steps_per_round):
+                inputs = [host_inputs(cfg, i, step) for i in range(cfg.K)]
+                if batched and not cfg.sparse:
+                    stacked = np.stack([inp["padded"] for inp in inputs])
+                    g = to_device(stacked.reshape(-1))
+                    keep.append(g)
+                    hp.hpsgd_local_step_all(g, stacked.shape[1] * stacked.itemsize)
+                else:
+                    for i, inp in enumerate(inputs):
+                        gpu_step(cfg, i, inp, keep)
+                for i, inp in enumerate(inputs):
+                    flat = inp["flat"]
+                    o.local_step(i, hashgen.bf16_to_f32(flat) if flat.dtype == np.uint16 else flat)
+                step += 1
+            hp.hpsgd_synchronize()
+            for i in range(cfg.K):
+                r, a = hp.hpsgd_get_replica(i)
+                assert_bitwise(gpu_flat(r, cfg), o.get_replica(i), "replica %d before sync %d" % (i, t))
+                assert_bitwise(gpu_flat(a, cfg), o.get_accumulated(i), "accumulated gradient %d before sync %d" % (i, t))
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+            hp.hpsgd_synchronize()
+            w, ghat, rs, accs = gpu_state(cfg)
+            assert_bitwise(w, o.get_global(), "global after sync %d" % t)
+            assert_bitwise(ghat, o.get_synced(), "AllReduce result after sync %d" % t)
+            for i in range(cfg.K):
+                assert_bitwise(rs[i], o.get_global(), "replica %d after sync %d" % (i, t))
+                assert not accs[i].any(), "accumulator %d not reset" % i
+        got = gpu_global(cfg)
+    want = o.get_global()
+    o.close()
+    return got, want

@@ -281,3 +281,41 @@ def test_fused_mixed_with_other_calls():
         w, D, rs, ms = gu.gpu_state(cfg)
         gu.assert_bitwise(w, o.get_global(), "global after back-to-back merges")
         gu.assert_bitwise(D, o.get_pending(), "pending change after back-to-back merges")
+
+
+# ---------------------------------------------------------------- Algorithms 2/3 as printed (accumulated gradients)
+@pytest.mark.parametrize("K,sizes,batched,chunks,H", [(4, [1_048_576], True, 1, 1), (2, [4], False, 1, 1),
+                                                      (16, [70_001, 33, 4096], True, 3, 1), (3, [5000, 77], False, 2, 3),
+                                                      (5, [129], False, 1, 2), (8, [300_000], True, 5, 1)])
+def test_gradient_accumulation_form(K, sizes, batched, chunks, H):
+    cfg = small("accum", K, sizes, T=4, lr=0.01, momentum=0.0, kind="uniform", scale=1e-2, seed=1)
+    got, want = gu.run_both_accum(cfg, cfg.T, batched=batched, chunks=chunks, steps_per_round=H)
+    assert gu.max_rel_err(got, want) <= 1e-6
+
+
+def test_gradient_accumulation_form_sparse_bf16():
+    cfg = small("accum_sparse", 4, [1000, 200 * 32, 55], T=3, lr=0.01, momentum=0.0, dtype="bf16",
+                sparse=(1, 200, 32), scale=1e-3)
+    gu.run_both_accum(cfg, cfg.T)
+
+
+def test_gradient_accumulation_form_agrees_with_replica_change_form():
+    """Eq. 1 == Eq. 2: both forms give the same global model up to rounding."""
+    cfg = small("forms", 8, [100_000], T=6, lr=0.01, momentum=0.0, kind="uniform", scale=1e-2, seed=1)
+    a, _ = gu.run_both_accum(cfg, cfg.T, batched=True)
+    b, _ = gu.run_both(cfg, cfg.T, batched=True)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-7)
+
+
+def test_gradient_accumulation_form_rejects_momentum():
+    hp.hpsgd_destroy()
+    hp.hpsgd_set_form(hp.HPSGD_FORM_GRADIENT_ACCUMULATION)
+    with pytest.raises(hp.HpsgdError) as err:
+        hp.hpsgd_init(1000, 2, 0.1, 0.9, 1)
+    assert err.value.code == hp.HPSGD_E_BADARG
+    hp.hpsgd_init(1000, 2, 0.1, 0.0, 1)
+    with pytest.raises(hp.HpsgdError):
+        hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, 1e-3)
+    hp.hpsgd_destroy()
+    with pytest.raises(hp.HpsgdError):
+        hp.hpsgd_set_form(7)
