@@ -319,3 +319,29 @@ def test_gradient_accumulation_form_rejects_momentum():
     hp.hpsgd_destroy()
     with pytest.raises(hp.HpsgdError):
         hp.hpsgd_set_form(7)
+
+
+# ---------------------------------------------------------------- Local SGD (Algorithm 1) and SSGD as modes
+@pytest.mark.parametrize("gamma", [1, 8])
+def test_local_sgd_and_ssgd_modes(gamma):
+    """staleness 0 with gamma plain-SGD local steps per merge is Algorithm 1 (the global model is
+    the mean of the K local models); gamma = 1 is synchronous SGD on the mean gradient."""
+    cfg = small("localsgd", 4, [20_000, 31], T=3, lr=0.01, momentum=0.0, kind="uniform", scale=1e-2, seed=9,
+                staleness=0)
+    w = cfg.initial_global().astype(np.float64)
+    with gu.session(cfg, staleness=0):
+        step = 0
+        for loop in range(cfg.T):
+            local = np.repeat(w[None, :], cfg.K, axis=0)
+            keep = []
+            for e in range(gamma):
+                for i in range(cfg.K):
+                    inp = gu.host_inputs(cfg, i, step)
+                    gu.gpu_step(cfg, i, inp, keep)
+                    local[i] -= np.float64(np.float32(cfg.lr)) * inp["flat"]
+                step += 1
+            hp.hpsgd_sync_merge()
+            hp.hpsgd_synchronize()
+            w = local.mean(axis=0)                      # AllReduce(model) / n, Algorithm 1
+            np.testing.assert_allclose(gu.gpu_global(cfg), w, rtol=0, atol=2e-7)
+    gu.run_both(cfg, cfg.T, staleness=0, steps_per_round=gamma)     # and bit-exact against the oracle
