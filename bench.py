@@ -283,7 +283,9 @@ def run_gpu(args, cfg):
     hp.hpsgd_destroy()
     if len(cfg.sizes) > 1:
         hp.hpsgd_set_layout(list(cfg.sizes))
-    nbytes = hp.hpsgd_arena_bytes(P_pad, K, hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0,
+    hp.hpsgd_set_pipeline(args.pipeline)
+    nbytes = hp.hpsgd_arena_bytes(P_pad, K, (hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0) |
+                                  (hp.HPSGD_ARENA_PIPELINE if args.pipeline else 0),
                                   cfg.sparse[1] if cfg.sparse else 0)
     arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
     base = arena.data_ptr() + (-arena.data_ptr()) % 256
@@ -295,7 +297,7 @@ def run_gpu(args, cfg):
     hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
     hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
     hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, args.chunks)
+    hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if args.pipeline else args.chunks)
     hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, args.fuse)
     if cfg.sparse:
         hp.hpsgd_set_sparse_segment(*cfg.sparse)
@@ -387,13 +389,16 @@ def run_gpu(args, cfg):
         grad_bytes += active * 4 - (K * rows_total - active) * cols * gsz
     state_bytes = K * P * (8 + (8 if cfg.momentum else 0))        # r (and m) read and written
     per_round = {"local_step_kernel": grad_bytes + state_bytes,
-                 "merge_kernel": merge_bytes_per_index(cfg) * P,
+                 # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
+                 "merge_kernel": (12 + (K + 2) * 4) * P if args.pipeline else merge_bytes_per_index(cfg) * P,
                  "merge_step_kernel": 16 * P + grad_bytes + state_bytes}
     kernels = {}
     for name, (ms, n) in prof.items():
         if n == 0:
             continue
-        per_launch = per_round[name] / args.chunks / (K if (args.per_worker and name == "local_step_kernel") else 1)
+        per_launch = per_round[name] / (1 if args.pipeline else args.chunks) / (K if (args.per_worker and name == "local_step_kernel") else 1)
+        if args.pipeline and name == "merge_kernel":
+            per_launch /= 2
         gbs = per_launch * n / (ms * 1e-3) / 1e9
         kernels[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms, "algorithmic_bytes_per_launch": per_launch,
                          "achieved": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
@@ -429,7 +434,9 @@ def run_gpu(args, cfg):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic (counter-hash gradients generated on the device, %d rounds cycled)" % nbuf,
             "config": workload_config(cfg, {
-                "schedule": {"overlap": args.overlap, "chunks": args.chunks, "fuse_merge_into_next_step": args.fuse,
+                "schedule": {"overlap": args.overlap, "chunks": args.chunks,
+                             "fuse_merge_into_next_step": 0 if args.pipeline else args.fuse,
+                             "pipelined_commit_reduce": args.pipeline,
                              "local_step_call": "per worker" if args.per_worker else "all K in one call"},
                 "l2": "inputs larger than L2 (state + gradients are tens of GB)",
                 "multi_gpu": "independent replicas, no inter-GPU exchange"}),
@@ -496,6 +503,8 @@ def main():
     ap.add_argument("--overlap", type=int, default=1)
     ap.add_argument("--chunks", type=int, default=1)
     ap.add_argument("--fuse", type=int, default=1, help="carry each merge into the next batched local step (one kernel)")
+    ap.add_argument("--pipeline", type=int, default=0,
+                    help="paper timeline: commit on the main stream, K-way reduce on the side stream, double-buffered replicas")
     ap.add_argument("--per-worker", action="store_true", help="K hpsgd_local_step calls instead of one batched call")
     ap.add_argument("--grad-buffers", type=int, default=2, help="rounds of device-resident gradients to cycle")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -74,7 +74,7 @@ enum { HPSGD_F32 = 0, HPSGD_BF16 = 1 };
 enum { HPSGD_GEN_UNIFORM = 0, HPSGD_GEN_GAUSS = 1 };
 
 /* Flags of hpsgd_arena_bytes. */
-enum { HPSGD_ARENA_MOMENTUM = 1 };
+enum { HPSGD_ARENA_MOMENTUM = 1, HPSGD_ARENA_PIPELINE = 2 };
 
 /* ------------------------------------------------------------------------------------
  * The four core calls.
@@ -156,12 +156,28 @@ int64_t hpsgd_layout_padded(int n_tensors, const int64_t* sizes, int64_t* offset
 enum { HPSGD_FORM_REPLICA_CHANGE = 0, HPSGD_FORM_GRADIENT_ACCUMULATION = 1 };
 int hpsgd_set_form(int form);
 
+/*
+ * Pipelined synchronisation for the next hpsgd_init (replica-change form, staleness 1, K <= 32),
+ * the paper's timeline (Fig. 1; Section 3.1: the synchronising process runs beside the training
+ * process).  hpsgd_sync_merge is split in two kernels: the commit w_next = w + D on the main
+ * stream, and the K-way reduce D = mean(r_i - w) of the period that just ended on the side
+ * stream.  Replicas and w are double-buffered (one more w and K more replica rows: set
+ * HPSGD_ARENA_PIPELINE when sizing an arena), and a worker's first local step of a period reads
+ * the new w instead of a re-cloned replica, so local steps never wait for the reduce; only the
+ * next hpsgd_sync_merge does.  Any number of local steps per period.  Same operations in the
+ * same order as the plain merge: results are bit-identical.  HPSGD_OPT_FUSE and
+ * HPSGD_OPT_CHUNKS do not apply.  The first pointer of hpsgd_get_replica is w itself for a
+ * worker that has not stepped since the last synchronisation.
+ */
+int hpsgd_set_pipeline(int enable);
+
 /* Declare the tensor sizes (host array, each > 0) used by the next hpsgd_init. */
 int hpsgd_set_layout(int n_tensors, const int64_t* sizes);
 
 /*
  * Bytes of device memory the state needs: w, D, K replicas, K momentum buffers when
- * flags has HPSGD_ARENA_MOMENTUM, plus the row->slot scratch map for a sparse-row
+ * flags has HPSGD_ARENA_MOMENTUM, a second w and K more replicas with HPSGD_ARENA_PIPELINE,
+ * plus the row->slot scratch map for a sparse-row
  * tensor of up to `sparse_rows` rows per worker (0 if unused) and a small table.
  */
 size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows);

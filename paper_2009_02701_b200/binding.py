@@ -19,6 +19,7 @@ HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP = 0, 1, 2
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
+HPSGD_ARENA_PIPELINE = 2
 HPSGD_FORM_REPLICA_CHANGE, HPSGD_FORM_GRADIENT_ACCUMULATION = 0, 1
 HPSGD_NOALLOC_MAX_ROWS = 262144
 
@@ -47,6 +48,7 @@ SIGNATURES = {
     "hpsgd_layout_padded": (_i64, [_ci, _P(_i64), _P(_i64)]),
     "hpsgd_set_layout": (_ci, [_ci, _P(_i64)]),
     "hpsgd_set_form": (_ci, [_ci]),
+    "hpsgd_set_pipeline": (_ci, [_ci]),
     "hpsgd_arena_bytes": (_sz, [_i64, _ci, _ci, _i64]),
     "hpsgd_bind": (_ci, [_vp, _sz, _vp, _vp]),
     "hpsgd_set_option": (_ci, [_ci, _f64]),
@@ -159,6 +161,10 @@ def hpsgd_set_layout(sizes):
 
 def hpsgd_set_form(form):
     return _check(load().hpsgd_set_form(int(form)))
+
+
+def hpsgd_set_pipeline(enable):
+    return _check(load().hpsgd_set_pipeline(int(enable)))
 
 
 def hpsgd_arena_bytes(P_pad, K, flags=0, sparse_rows=0):

@@ -60,6 +60,7 @@ struct Pending {                // configuration collected before hpsgd_init
     cudaStream_t main = nullptr, side = nullptr;
     bool have_streams = false;
     int form = HPSGD_FORM_REPLICA_CHANGE;
+    int pipeline = 0;
 } g_pending;
 
 struct Ctx {
@@ -86,6 +87,13 @@ struct Ctx {
     int64_t merges = 0;
     int form = HPSGD_FORM_REPLICA_CHANGE;  // what the workers carry: replica change or accumulated gradients
     int fuse = 0;                          // carry a merge into the next batched local step
+    int pipeline = 0;                      // commit/reduce split on double-buffered replicas
+    float* wbuf[2] = {nullptr, nullptr};   // pipeline: global model of the current / other period
+    float* rbuf[2] = {nullptr, nullptr};   // pipeline: replica sets of the current / other period
+    int cur = 0;                           // pipeline: which buffers the current period trains on
+    std::vector<char> touched;             // pipeline: worker has made a local step this period
+    cudaEvent_t ev_commit = nullptr, ev_reduce = nullptr;
+    bool reduce_outstanding = false;
     bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
     int deferred_flags = 0;
     int64_t launches = 0;
@@ -120,12 +128,12 @@ int64_t layout_of(const std::vector<int64_t>& sizes, std::vector<int64_t>* offse
     return pos;
 }
 
-// Regions of the arena, in order: w | D | r[K] | m[K] | table | slot maps (the rest).
+// Regions of the arena, in order: w | D | r[K] | m[K] | w2 | r2[K] | table | slot maps (the rest).
 struct ArenaPlan {
-    size_t w, D, r, m, table, slot, fixed;
+    size_t w, D, r, m, w2, r2, table, slot, fixed;
 };
 
-ArenaPlan plan_arena(int64_t stride, int K, bool momentum)
+ArenaPlan plan_arena(int64_t stride, int K, bool momentum, bool pipeline)
 {
     ArenaPlan a{};
     const size_t row = (size_t)stride * 4;
@@ -134,6 +142,8 @@ ArenaPlan plan_arena(int64_t stride, int K, bool momentum)
     a.D = pos; pos += row;
     a.r = pos; pos += row * K;
     a.m = pos; if (momentum) pos += row * K;
+    a.w2 = pos; if (pipeline) pos += row;
+    a.r2 = pos; if (pipeline) pos += row * K;
     a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kAlignBytes);
     a.slot = pos;
     a.fixed = pos;
@@ -253,6 +263,15 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
 {
     LocalLaunch L{};
     L.w0 = w0; L.nw = nw; L.gp = gp;
+    if (g.pipeline) {
+        // first step of a worker in this period: its replica is still the clone, i.e. w itself
+        for (int i = 0; i < nw; ++i) {
+            if (!g.touched[w0 + i]) {
+                L.gp.r_src[i] = g.w;
+                g.touched[w0 + i] = 1;
+            }
+        }
+    }
     L.p = StepParams{-g.lr, g.beta, g.lambda};
     L.seg = SparseSeg{0, 0, 1};
     if (sparse) {
@@ -351,10 +370,15 @@ int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; block
     const size_t row = (size_t)g.stride * 4;
     CUDA_TRY(cudaMemsetAsync(g.D, 0, row, g.main));
     if (g.m) CUDA_TRY(cudaMemsetAsync(g.m, 0, row * g.K, g.main));
-    const int64_t nvec = g.P_pad / 4;
-    clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
-    ++g.launches;
-    CUDA_TRY(cudaGetLastError());
+    if (g.pipeline) {
+        std::fill(g.touched.begin(), g.touched.end(), 0);      // replicas are w until their first step
+        g.reduce_outstanding = false;
+    } else {
+        const int64_t nvec = g.P_pad / 4;
+        clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
+        ++g.launches;
+        CUDA_TRY(cudaGetLastError());
+    }
     CUDA_TRY(cudaStreamSynchronize(g.main));
     g.D_valid = false;
     g.merges = 0;
@@ -414,6 +438,8 @@ void release_all()
     for (EventPair& ep : g.prof) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
     for (cudaEvent_t e : g.ev_local) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : g.ev_merge) if (e) cudaEventDestroy(e);
+    if (g.ev_commit) cudaEventDestroy(g.ev_commit);
+    if (g.ev_reduce) cudaEventDestroy(g.ev_reduce);
     for (int b = 0; b < 2; ++b) {
         if (g.stage[b]) cudaFree(g.stage[b]);
         if (g.stage_copied[b]) cudaEventDestroy(g.stage_copied[b]);
@@ -478,6 +504,53 @@ int enqueue_merge(int flags)
             g.merge_unwaited[c] = 1;
         }
     }
+    return check_async();
+}
+
+template <int KT>
+void launch_reduce(const float* w_old, const ReducePtrs& rp, int64_t n)
+{
+    reduce_kernel<KT><<<hot_grid(n), kHotThreads, 0, g.side>>>(w_old, g.D, rp, g.K, n);
+}
+
+// Pipelined synchronisation: the commit w_next = w + D runs on the main stream, in order with
+// the local steps; the K-way reduce of the period that just ended runs on the side stream and
+// nothing on the main stream waits for it until the NEXT synchronisation needs its result.
+int enqueue_pipelined_merge(int flags)
+{
+    const int64_t n = g.P_pad / 8;
+    const int nxt = g.cur ^ 1;
+    if (g.reduce_outstanding) {
+        // the previous reduce still reads the buffers about to be written and produces the D read here
+        CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_reduce, 0));
+        g.reduce_outstanding = false;
+    }
+    EventPair ep{};
+    TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE, &ep));
+    commit_kernel<<<hot_grid(n), kHotThreads, 0, g.main>>>(g.wbuf[g.cur], g.D, g.wbuf[nxt], n, flags);
+    ++g.launches;
+    TRY(prof_end(g.main, &ep));
+    CUDA_TRY(cudaEventRecord(g.ev_commit, g.main));
+    CUDA_TRY(cudaStreamWaitEvent(g.side, g.ev_commit, 0));
+    ReducePtrs rp{};
+    for (int i = 0; i < g.K; ++i)
+        rp.src[i] = g.touched[i] ? g.rbuf[g.cur] + (int64_t)i * g.stride : g.wbuf[g.cur];
+    EventPair ep2{};
+    TRY(prof_begin(g.side, HPSGD_KERNEL_MERGE, &ep2));
+    switch (g.K) {
+    case 4: launch_reduce<4>(g.wbuf[g.cur], rp, n); break;
+    case 8: launch_reduce<8>(g.wbuf[g.cur], rp, n); break;
+    case 16: launch_reduce<16>(g.wbuf[g.cur], rp, n); break;
+    default: launch_reduce<0>(g.wbuf[g.cur], rp, n); break;
+    }
+    ++g.launches;
+    TRY(prof_end(g.side, &ep2));
+    CUDA_TRY(cudaEventRecord(g.ev_reduce, g.side));
+    g.reduce_outstanding = true;
+    g.cur = nxt;
+    g.w = g.wbuf[nxt];
+    g.r = g.rbuf[nxt];
+    std::fill(g.touched.begin(), g.touched.end(), 0);
     return check_async();
 }
 
@@ -596,6 +669,14 @@ int hpsgd_set_form(int form)
     return HPSGD_OK;
 }
 
+int hpsgd_set_pipeline(int enable)
+{
+    if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_set_pipeline must precede hpsgd_init");
+    if (enable != 0 && enable != 1) return fail(HPSGD_E_BADARG, "enable must be 0 or 1");
+    g_pending.pipeline = enable;
+    return HPSGD_OK;
+}
+
 int hpsgd_set_layout(int n_tensors, const int64_t* sizes)
 {
     if (g.inited) return fail(HPSGD_E_STATE, "hpsgd_set_layout must precede hpsgd_init");
@@ -610,7 +691,8 @@ size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows)
     if (P_pad <= 0 || K <= 0 || sparse_rows < 0) return 0;
     const int64_t stride = (P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
     const int64_t cap = (sparse_rows + 63) / 64 * 64;
-    return plan_arena(stride, K, (flags & HPSGD_ARENA_MOMENTUM) != 0).fixed + (size_t)cap * 4 * K;
+    return plan_arena(stride, K, (flags & HPSGD_ARENA_MOMENTUM) != 0, (flags & HPSGD_ARENA_PIPELINE) != 0).fixed +
+           (size_t)cap * 4 * K;
 }
 
 int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream)
@@ -642,6 +724,10 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     if (!(momentum >= 0.f && momentum < 1.f)) return fail(HPSGD_E_BADARG, "momentum must be in [0, 1)");
     if (g_pending.form == HPSGD_FORM_GRADIENT_ACCUMULATION && momentum != 0.f)
         return fail(HPSGD_E_BADARG, "the gradient-accumulation form is the paper's plain SGD: momentum must be 0");
+    if (g_pending.pipeline && g_pending.form != HPSGD_FORM_REPLICA_CHANGE)
+        return fail(HPSGD_E_BADARG, "the pipelined schedule is implemented for the replica-change form");
+    if (g_pending.pipeline && K > kMaxBatch)
+        return fail(HPSGD_E_UNSUPPORTED, "the pipelined schedule supports K <= %d", kMaxBatch);
     std::vector<int64_t> sizes = g_pending.sizes;
     if (sizes.empty()) sizes.push_back(P);
     int64_t sum = 0;
@@ -665,7 +751,8 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.stride = (g.P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
     g.form = g_pending.form;
     const bool mom = momentum != 0.f || g.form == HPSGD_FORM_GRADIENT_ACCUMULATION;   // K extra rows: m_i or a_i
-    const ArenaPlan a = plan_arena(g.stride, K, mom);
+    g.pipeline = g_pending.pipeline;
+    const ArenaPlan a = plan_arena(g.stride, K, mom, g.pipeline != 0);
 
     if (g_pending.arena) {
         if (g_pending.arena_bytes < a.fixed) {
@@ -693,6 +780,13 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.r = reinterpret_cast<float*>(g.arena + a.r);
     g.m = mom ? reinterpret_cast<float*>(g.arena + a.m) : nullptr;
     g.d_table = reinterpret_cast<int64_t*>(g.arena + a.table);
+    g.wbuf[0] = g.w;
+    g.rbuf[0] = g.r;
+    if (g.pipeline) {
+        g.wbuf[1] = reinterpret_cast<float*>(g.arena + a.w2);
+        g.rbuf[1] = reinterpret_cast<float*>(g.arena + a.r2);
+        g.touched.assign(K, 0);
+    }
 
     if (g_pending.have_streams) {
         g.main = g_pending.main;
@@ -708,6 +802,11 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.inited = true;
     int rc = make_chunk_events(1);
     if (rc) { release_all(); return rc; }
+    if (g.pipeline && (cudaEventCreateWithFlags(&g.ev_commit, cudaEventDisableTiming) != cudaSuccess ||
+                       cudaEventCreateWithFlags(&g.ev_reduce, cudaEventDisableTiming) != cudaSuccess)) {
+        release_all();
+        return fail(HPSGD_E_CUDA, "could not create events");
+    }
 
     // device table: offsets | starts | sizes
     const size_t n = sizes.size();
@@ -763,6 +862,8 @@ int hpsgd_set_option(int key, double value)
     case HPSGD_OPT_STALENESS:
         if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "staleness must be 0 or 1");
         if (g.merges) return fail(HPSGD_E_STATE, "staleness can only change before the first merge");
+        if (value == 0.0 && g.pipeline)
+            return fail(HPSGD_E_BADARG, "the pipelined schedule needs the one-synchronisation delay (staleness 1)");
         g.staleness = (int)value;
         return HPSGD_OK;
     case HPSGD_OPT_GRAD_DTYPE:
@@ -779,6 +880,7 @@ int hpsgd_set_option(int key, double value)
     case HPSGD_OPT_CHUNKS:
         if (!(value >= 1.0 && value <= kMaxChunks && value == (double)(int)value))
             return fail(HPSGD_E_BADARG, "chunks must be an integer in [1, %d]", kMaxChunks);
+        if (value != 1.0 && g.pipeline) return fail(HPSGD_E_BADARG, "the pipelined schedule is not cut into chunks");
         TRY(sync_all());
         return make_chunk_events((int)value);
     case HPSGD_OPT_FUSE:
@@ -936,6 +1038,7 @@ int hpsgd_sync_merge(void)
     else if (g.D_valid) flags |= kMergeApplyPending;
     g.D_valid = true;
     g.merges += 1;
+    if (g.pipeline) return enqueue_pipelined_merge(flags);
     if (g.fuse && g.form == HPSGD_FORM_REPLICA_CHANGE) {
         g.merge_deferred = true;
         g.deferred_flags = flags;
@@ -990,7 +1093,7 @@ int hpsgd_get_replica(int worker, const float** r, const float** m)
 {
     TRY(need_init());
     TRY(check_worker(worker));
-    if (r) *r = g.r + (int64_t)worker * g.stride;
+    if (r) *r = (g.pipeline && !g.touched[worker]) ? g.w : g.r + (int64_t)worker * g.stride;
     if (m) *m = g.m ? g.m + (int64_t)worker * g.stride : nullptr;
     return HPSGD_OK;
 }

@@ -146,6 +146,9 @@ struct BatchPtrs {
     const void* dense[kMaxBatch];
     const void* row_vals[kMaxBatch];
     const int32_t* slot[kMaxBatch];
+    const float* r_src[kMaxBatch];   // where the worker's replica is READ from; NULL: its own row.
+                                     // (pipelined schedule: the first step after a synchronisation
+                                     // reads the global model, which is the not-yet-written clone)
 };
 
 // One worker per blockIdx.y; workers' replicas/momenta are `stride` floats apart starting
@@ -167,8 +170,9 @@ local_step_kernel(float* __restrict__ r_base, float* __restrict__ m_base, int64_
     const int32_t* __restrict__ slot = SPARSE ? gp.slot[wk] : nullptr;
 
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    const float* __restrict__ rs = gp.r_src[wk] ? gp.r_src[wk] : r;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
-        f8 rr = ld8(r + o * 8);
+        f8 rr = ld8(rs + o * 8);
         f8 mm;
         if (MOM) mm = ld8(m + o * 8);
         f8 gg;
@@ -277,6 +281,77 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
         const int Kn = KT > 0 ? KT : K;
 #pragma unroll 4
         for (int i = 0; i < Kn; ++i) st8(r + (int64_t)i * stride + e, wn);
+    }
+}
+
+// ---------------------------------------------------------------------------- pipelined synchronisation
+// The paper's timeline (Fig. 1): the synchronising process first commits the previous
+// AllReduce result, then all-reduces while the training process already works on replicas
+// cloned from the updated global model.  The merge is therefore split in two:
+//   commit:  w_next = w + D          (D from the previous synchronisation, if any)
+//   reduce:  D = ((r_0 - w) + ... + (r_{K-1} - w)) / K     over the replicas of the period that
+//            just ended and the w they were cloned from,
+// with replicas and w double-buffered so that the reduce and the next period's local steps
+// touch different memory.  Same operations and order as merge_kernel.
+__global__ void __launch_bounds__(kHotThreads)
+commit_kernel(const float* __restrict__ w, const float* __restrict__ D, float* __restrict__ w_next,
+              int64_t n, int flags)
+{
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
+        f8 wv = ld8(w + o * 8);
+        if (flags & kMergeApplyPending) {
+            const f8 dv = ld8(D + o * 8);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) wv.v[q] = __fadd_rn(wv.v[q], dv.v[q]);
+        }
+        st8(w_next + o * 8, wv);
+    }
+}
+
+// Per-worker source of the reduce: the worker's replica, or w itself for a worker that made
+// no local step in the period (its change is r - w = 0).
+struct ReducePtrs {
+    const float* src[kMaxBatch];
+};
+
+template <int KT>
+__global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
+reduce_kernel(const float* __restrict__ w, float* __restrict__ D, ReducePtrs rp, int K, int64_t n)
+{
+    const int Kn = KT > 0 ? KT : K;
+    const float fK = (float)Kn;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
+        const int64_t e = o * 8;
+        const f8 wv = ld8(w + e);
+        f8 acc;
+        if constexpr (KT > 0) {
+            f8 rv[KT];
+#pragma unroll
+            for (int i = 0; i < KT; ++i) rv[i] = ld8(rp.src[i] + e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(rv[0].v[q], wv.v[q]);
+#pragma unroll
+            for (int i = 1; i < KT; ++i)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
+        } else {
+            {
+                const f8 r0 = ld8(rp.src[0] + e);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
+            }
+            for (int i = 1; i < K; ++i) {
+                const f8 ri = ld8(rp.src[i] + e);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
+            }
+        }
+        f8 dnew;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) dnew.v[q] = __fdiv_rn(acc.v[q], fK);
+        st8(D + e, dnew);
     }
 }
 

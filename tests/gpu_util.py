@@ -35,7 +35,8 @@ def to_device(a: np.ndarray) -> torch.Tensor:
 
 
 @contextlib.contextmanager
-def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, lend_arena=False, streams=False, canary=False):
+def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, pipeline=0, lend_arena=False, streams=False,
+            canary=False):
     """hpsgd_init for a workload (layout, options, optional lent arena/streams); destroys on exit."""
     hp.hpsgd_destroy()
     lay = cfg.layout
@@ -43,11 +44,13 @@ def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, lend_ar
     if len(cfg.sizes) > 1:
         hp.hpsgd_set_layout(list(cfg.sizes))
     hp.hpsgd_set_form(form)
+    hp.hpsgd_set_pipeline(pipeline)
     if lend_arena or streams:
         arena, nbytes, main, side = None, 0, None, None
         if lend_arena:
             rows = cfg.sparse[1] if cfg.sparse else 0
-            nbytes = hp.hpsgd_arena_bytes(lay.P_pad, cfg.K, hp.HPSGD_ARENA_MOMENTUM if (cfg.momentum or form) else 0, rows)
+            flags = (hp.HPSGD_ARENA_MOMENTUM if (cfg.momentum or form) else 0) | (hp.HPSGD_ARENA_PIPELINE if pipeline else 0)
+            nbytes = hp.hpsgd_arena_bytes(lay.P_pad, cfg.K, flags, rows)
             guard = 4096 if canary else 0
             buf = torch.full((nbytes + 2 * guard + 256,), 0xA5, dtype=torch.uint8, device=DEV)
             base = buf.data_ptr() + guard
@@ -176,11 +179,12 @@ def max_rel_err(got, want, floor=1e-6):
     return float(np.max(np.abs(got - want) / np.maximum(np.abs(want), floor)))
 
 
-def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, fuse=0, batched=False, steps_per_round=1,
+def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, fuse=0, pipeline=0, batched=False, steps_per_round=1,
              skip_worker=None, session_kw=None, check_each_round=False):
     """Run T rounds on the GPU and on the oracle with host-generated inputs; compare bitwise."""
     o = oracle_for(cfg, staleness)
-    with session(cfg, staleness=staleness, overlap=overlap, chunks=chunks, fuse=fuse, **(session_kw or {})):
+    with session(cfg, staleness=staleness, overlap=overlap, chunks=chunks, fuse=fuse, pipeline=pipeline,
+                 **(session_kw or {})):
         assert_bitwise(gpu_global(cfg), o.get_global(), "initial global model")
         step = 0
         alive = []
@@ -218,8 +222,8 @@ def run_both(cfg, T, *, staleness=None, overlap=1, chunks=1, fuse=0, batched=Fal
                 w, D, rs, ms = gpu_state(cfg)
                 assert_bitwise(w, o.get_global(), "global after merge %d" % t)
                 assert_bitwise(D, o.get_pending(), "pending change after merge %d" % t)
-            if fuse:
-                alive.append(keep)          # no synchronise here: it would launch the deferred merge
+            if fuse or pipeline:
+                alive.append(keep)          # no synchronise here: keep the merge and the next steps in flight
             else:
                 hp.hpsgd_synchronize()
                 del keep

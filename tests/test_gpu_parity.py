@@ -345,3 +345,39 @@ def test_local_sgd_and_ssgd_modes(gamma):
             w = local.mean(axis=0)                      # AllReduce(model) / n, Algorithm 1
             np.testing.assert_allclose(gu.gpu_global(cfg), w, rtol=0, atol=2e-7)
     gu.run_both(cfg, cfg.T, staleness=0, steps_per_round=gamma)     # and bit-exact against the oracle
+
+
+# ---------------------------------------------------------------- pipelined synchronisation (the paper's timeline)
+@pytest.mark.parametrize("K,momentum,wd,H,batched", [(16, 0.9, 0.0, 1, True), (8, 0.9, 5e-4, 3, False), (4, 0.0, 0.0, 1, False),
+                                                     (3, 0.9, 0.0, 2, True), (5, 0.0, 1e-3, 1, True), (1, 0.9, 0.0, 1, False)])
+def test_pipelined_sync_matches_oracle(K, momentum, wd, H, batched):
+    cfg = small("pipe", K, [70_001, 33, 4096], T=5, momentum=momentum, wd=wd)
+    gu.run_both(cfg, cfg.T, pipeline=1, batched=batched, steps_per_round=H)
+    gu.run_both(cfg, 3, pipeline=1, batched=batched, steps_per_round=H, check_each_round=True,
+                session_kw=dict(lend_arena=True, canary=True, streams=True))
+
+
+def test_pipelined_sync_idle_worker_and_sparse_rows():
+    cfg = small("pipe_skip", 4, [3000], T=4)
+    gu.run_both(cfg, cfg.T, pipeline=1, skip_worker=2, check_each_round=True)
+    cfg = small("pipe_sparse", 5, [1000, 300 * 64, 777, 64], T=4, dtype="bf16", sparse=(1, 300, 64), scale=1e-3)
+    gu.run_both(cfg, cfg.T, pipeline=1, batched=True)
+    gu.run_both(cfg, cfg.T, pipeline=1, batched=False)
+
+
+def test_pipelined_sync_argument_checks():
+    hp.hpsgd_destroy()
+    hp.hpsgd_set_pipeline(1)
+    hp.hpsgd_set_form(hp.HPSGD_FORM_GRADIENT_ACCUMULATION)
+    with pytest.raises(hp.HpsgdError):
+        hp.hpsgd_init(1000, 2, 0.1, 0.0, 1)
+    hp.hpsgd_destroy()
+    hp.hpsgd_set_pipeline(1)
+    with pytest.raises(hp.HpsgdError) as err:
+        hp.hpsgd_init(1000, 33, 0.1, 0.0, 1)
+    assert err.value.code == hp.HPSGD_E_UNSUPPORTED
+    hp.hpsgd_init(1000, 4, 0.1, 0.0, 1)
+    for key, val in ((hp.HPSGD_OPT_STALENESS, 0), (hp.HPSGD_OPT_CHUNKS, 4)):
+        with pytest.raises(hp.HpsgdError):
+            hp.hpsgd_set_option(key, val)
+    hp.hpsgd_destroy()
