@@ -304,6 +304,19 @@ int hpsgd_copy_global(float* host_out, int64_t n);
 int hpsgd_get_replica(int worker, const float** r, const float** m);
 int hpsgd_get_pending(const float** D);
 
+/*
+ * Checkpoint of the optimisation state (the paper has none; a long run needs one): a HOST blob
+ * holding w, D, every replica, every momentum (or accumulated-gradient) buffer in the flat
+ * layout, the merge count and whether a pending change exists.  Hyper-parameters and options
+ * are not part of it: import into a state initialised with the same P, layout, K, form and
+ * momentum on/off (else HPSGD_E_BADARG), then set the options again.  Both calls wait for all
+ * enqueued work (a merge deferred by HPSGD_OPT_FUSE is launched first) and block.  A run of T
+ * rounds and a run of T/2 rounds + export + import + T/2 rounds give bit-identical states.
+ */
+size_t hpsgd_state_bytes(void);                                   /* 0 before hpsgd_init */
+int hpsgd_export_state(void* host_out, size_t bytes);
+int hpsgd_import_state(const void* host_in, size_t bytes);
+
 /* Current sizes: any out pointer may be NULL. */
 int hpsgd_get_sizes(int64_t* P, int64_t* P_pad, int* K, int64_t* merges);
 

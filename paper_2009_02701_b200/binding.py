@@ -63,6 +63,9 @@ SIGNATURES = {
     "hpsgd_copy_global": (_ci, [_vp, _i64]),
     "hpsgd_get_replica": (_ci, [_ci, _P(_vp), _P(_vp)]),
     "hpsgd_get_pending": (_ci, [_P(_vp)]),
+    "hpsgd_state_bytes": (_sz, []),
+    "hpsgd_export_state": (_ci, [_vp, _sz]),
+    "hpsgd_import_state": (_ci, [_vp, _sz]),
     "hpsgd_get_sizes": (_ci, [_P(_i64), _P(_i64), _P(_ci), _P(_i64)]),
     "hpsgd_tensor_offset": (_i64, [_ci]),
     "hpsgd_gen_grads": (_ci, [_vp, _ci, _ci, _ci, _f64]),
@@ -235,6 +238,19 @@ def hpsgd_get_pending():
     d = _vp()
     _check(load().hpsgd_get_pending(ctypes.byref(d)))
     return d.value
+
+
+def hpsgd_state_bytes():
+    return int(load().hpsgd_state_bytes())
+
+
+def hpsgd_export_state(host_buf):
+    """host_buf: a writable host buffer (e.g. numpy uint8 array) of hpsgd_state_bytes() bytes."""
+    return _check(load().hpsgd_export_state(_ptr(host_buf), int(host_buf.nbytes)))
+
+
+def hpsgd_import_state(host_buf):
+    return _check(load().hpsgd_import_state(_ptr(host_buf), int(host_buf.nbytes)))
 
 
 def hpsgd_get_sizes():

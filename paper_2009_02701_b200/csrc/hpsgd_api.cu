@@ -1105,6 +1105,92 @@ int hpsgd_get_pending(const float** D)
     return HPSGD_OK;
 }
 
+// ------------------------------------------------------------------------- checkpoint
+namespace {
+
+struct StateHeader {
+    uint64_t magic;            // "HPSGDST1"
+    int64_t P, P_pad, merges;
+    int32_t K, form, has_aux, staleness, D_valid, reserved;
+};
+constexpr uint64_t kStateMagic = 0x3154534447535048ULL;
+
+size_t state_bytes()
+{
+    const size_t row = (size_t)g.P_pad * 4;
+    return sizeof(StateHeader) + row * (2 + (size_t)g.K * (g.m ? 2 : 1));
+}
+
+}  // namespace
+
+size_t hpsgd_state_bytes(void)
+{
+    if (!g.inited) return 0;
+    return state_bytes();
+}
+
+int hpsgd_export_state(void* host_out, size_t bytes)
+{
+    TRY(need_init());
+    if (!host_out || bytes < state_bytes()) return fail(HPSGD_E_BADARG, "need a host buffer of hpsgd_state_bytes() = %zu bytes", state_bytes());
+    TRY(flush_deferred());
+    TRY(sync_all());
+    StateHeader h{};
+    h.magic = kStateMagic;
+    h.P = g.P; h.P_pad = g.P_pad; h.merges = g.merges;
+    h.K = g.K; h.form = g.form; h.has_aux = g.m ? 1 : 0; h.staleness = g.staleness; h.D_valid = g.D_valid ? 1 : 0;
+    char* out = static_cast<char*>(host_out);
+    std::memcpy(out, &h, sizeof h);
+    out += sizeof h;
+    const size_t row = (size_t)g.P_pad * 4;
+    CUDA_TRY(cudaMemcpy(out, g.w, row, cudaMemcpyDeviceToHost)); out += row;
+    CUDA_TRY(cudaMemcpy(out, g.D, row, cudaMemcpyDeviceToHost)); out += row;
+    for (int i = 0; i < g.K; ++i) {
+        // pipelined schedule: a worker that has not stepped since the last synchronisation has w as its replica
+        const float* src = (g.pipeline && !g.touched[i]) ? g.w : g.r + (int64_t)i * g.stride;
+        CUDA_TRY(cudaMemcpy(out, src, row, cudaMemcpyDeviceToHost)); out += row;
+    }
+    if (g.m)
+        for (int i = 0; i < g.K; ++i) {
+            CUDA_TRY(cudaMemcpy(out, g.m + (int64_t)i * g.stride, row, cudaMemcpyDeviceToHost)); out += row;
+        }
+    return HPSGD_OK;
+}
+
+int hpsgd_import_state(const void* host_in, size_t bytes)
+{
+    TRY(need_init());
+    if (!host_in || bytes < sizeof(StateHeader)) return fail(HPSGD_E_BADARG, "state blob too short");
+    StateHeader h;
+    std::memcpy(&h, host_in, sizeof h);
+    if (h.magic != kStateMagic) return fail(HPSGD_E_BADARG, "not a state blob of this library");
+    if (h.P != g.P || h.P_pad != g.P_pad || h.K != g.K || h.form != g.form || h.has_aux != (g.m ? 1 : 0))
+        return fail(HPSGD_E_BADARG, "state blob does not match the initialised sizes, form or optimiser");
+    if (bytes < state_bytes()) return fail(HPSGD_E_BADARG, "state blob truncated");
+    if (h.staleness != g.staleness && g.merges) return fail(HPSGD_E_STATE, "staleness differs and merges have already run");
+    TRY(flush_deferred());
+    TRY(sync_all());
+    const char* in = static_cast<const char*>(host_in) + sizeof h;
+    const size_t row = (size_t)g.P_pad * 4;
+    CUDA_TRY(cudaMemcpy(g.w, in, row, cudaMemcpyHostToDevice)); in += row;
+    CUDA_TRY(cudaMemcpy(g.D, in, row, cudaMemcpyHostToDevice)); in += row;
+    for (int i = 0; i < g.K; ++i) {
+        CUDA_TRY(cudaMemcpy(g.r + (int64_t)i * g.stride, in, row, cudaMemcpyHostToDevice)); in += row;
+    }
+    if (g.m)
+        for (int i = 0; i < g.K; ++i) {
+            CUDA_TRY(cudaMemcpy(g.m + (int64_t)i * g.stride, in, row, cudaMemcpyHostToDevice)); in += row;
+        }
+    g.staleness = h.staleness;
+    g.D_valid = h.D_valid != 0;
+    g.merges = h.merges;
+    if (g.pipeline) std::fill(g.touched.begin(), g.touched.end(), 1);   // every replica row now holds real data
+    g.reduce_outstanding = false;
+    std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
+    std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
+    return HPSGD_OK;
+}
+
 int hpsgd_get_sizes(int64_t* P, int64_t* P_pad, int* K, int64_t* merges)
 {
     TRY(need_init());

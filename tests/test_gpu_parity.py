@@ -381,3 +381,41 @@ def test_pipelined_sync_argument_checks():
         with pytest.raises(hp.HpsgdError):
             hp.hpsgd_set_option(key, val)
     hp.hpsgd_destroy()
+
+
+# ---------------------------------------------------------------- checkpoint
+@pytest.mark.parametrize("mode", ["plain", "fuse", "pipeline", "accum"])
+def test_export_import_resumes_bit_identically(mode):
+    momentum = 0.0 if mode == "accum" else 0.9
+    cfg = small("ckpt", 4, [20_000, 77], T=6, momentum=momentum, lr=0.05)
+    kw = dict(fuse=int(mode == "fuse"), pipeline=int(mode == "pipeline"),
+              form=hp.HPSGD_FORM_GRADIENT_ACCUMULATION if mode == "accum" else 0)
+
+    def rounds(t0, t1, keep):
+        for t in range(t0, t1):
+            stacked = np.stack([gu.host_inputs(cfg, i, t)["padded"] for i in range(cfg.K)])
+            keep.append(gu.to_device(stacked.reshape(-1)))
+            hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
+            hp.hpsgd_sync_merge()
+
+    with gu.session(cfg, **kw):
+        keep = []
+        rounds(0, cfg.T, keep)
+        straight = gu.gpu_state(cfg)
+    with gu.session(cfg, **kw):
+        keep = []
+        rounds(0, 3, keep)
+        blob = np.empty(hp.hpsgd_state_bytes(), dtype=np.uint8)
+        hp.hpsgd_export_state(blob)
+    with gu.session(cfg, **kw):
+        with pytest.raises(hp.HpsgdError):
+            hp.hpsgd_import_state(blob[:100])
+        hp.hpsgd_import_state(blob)
+        assert hp.hpsgd_get_sizes()[3] == 3
+        keep = []
+        rounds(3, cfg.T, keep)
+        resumed = gu.gpu_state(cfg)
+    gu.assert_bitwise(resumed[0], straight[0], "global model after resume")
+    gu.assert_bitwise(resumed[1], straight[1], "pending change after resume")
+    for a, b in zip(resumed[2] + resumed[3], straight[2] + straight[3]):
+        gu.assert_bitwise(a, b, "replica / momentum after resume")
