@@ -419,3 +419,11 @@ def test_export_import_resumes_bit_identically(mode):
     gu.assert_bitwise(resumed[1], straight[1], "pending change after resume")
     for a, b in zip(resumed[2] + resumed[3], straight[2] + straight[3]):
         gu.assert_bitwise(a, b, "replica / momentum after resume")
+
+
+def test_more_workers_than_one_batched_launch_addresses():
+    """K = 40 > 32: batched calls are issued in groups of 32 workers, the fused path steps aside."""
+    cfg = small("k40", 40, [5000, 33], T=3, momentum=0.9)
+    gu.run_both(cfg, cfg.T, batched=True)
+    gu.run_both(cfg, cfg.T, batched=True, fuse=1, chunks=2)
+    gu.run_both(cfg, cfg.T, batched=False)
