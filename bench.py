@@ -279,28 +279,32 @@ def run_gpu(args, cfg):
     gsz = 2 if bf16 else 4
     kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
 
-    # ---- state: arena and streams come from torch, the library only computes
-    hp.hpsgd_destroy()
-    if len(cfg.sizes) > 1:
-        hp.hpsgd_set_layout(list(cfg.sizes))
-    hp.hpsgd_set_pipeline(args.pipeline)
-    nbytes = hp.hpsgd_arena_bytes(P_pad, K, (hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0) |
-                                  (hp.HPSGD_ARENA_PIPELINE if args.pipeline else 0),
+    # ---- state: arena and streams come from torch, the library only computes.  The arena is
+    # sized for the pipelined schedule too, so that every schedule can be timed in one run.
+    nbytes = hp.hpsgd_arena_bytes(P_pad, K, (hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0) | hp.HPSGD_ARENA_PIPELINE,
                                   cfg.sparse[1] if cfg.sparse else 0)
     arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
     base = arena.data_ptr() + (-arena.data_ptr()) % 256
     main, side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-    hp.hpsgd_bind(base, nbytes, main, side)
-    hp.hpsgd_init(P, K, cfg.lr, cfg.momentum, cfg.seed)
-    if cfg.weight_decay:
-        hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, cfg.weight_decay)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if args.pipeline else args.chunks)
-    hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, args.fuse)
-    if cfg.sparse:
-        hp.hpsgd_set_sparse_segment(*cfg.sparse)
+
+    def setup(pipeline, fuse, chunks):
+        hp.hpsgd_destroy()
+        if len(cfg.sizes) > 1:
+            hp.hpsgd_set_layout(list(cfg.sizes))
+        hp.hpsgd_set_pipeline(pipeline)
+        hp.hpsgd_bind(base, nbytes, main, side)
+        hp.hpsgd_init(P, K, cfg.lr, cfg.momentum, cfg.seed)
+        if cfg.weight_decay:
+            hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, cfg.weight_decay)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if pipeline else chunks)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
+        if cfg.sparse:
+            hp.hpsgd_set_sparse_segment(*cfg.sparse)
+
+    setup(args.pipeline, args.fuse, args.chunks)
 
     # ---- inputs: `nbuf` rounds of gradients for all K workers, generated on the device
     nbuf = args.grad_buffers
@@ -416,6 +420,30 @@ def run_gpu(args, cfg):
     unfused_round = per_round["local_step_kernel"] + per_round["merge_kernel"]
     roofline["round_unfused_equivalent"] = unfused_round * args.steps / (elapsed_ms * 1e-3) / 1e9
 
+    # ---- the other schedules of the same path, timed briefly the same way (same inputs, same work)
+    other = {}
+    if args.other_schedule_steps > 0 and not args.per_worker:
+        for name, pipe, fuse in (("separate merge and local-step kernels on two streams", 0, 0),
+                                 ("pipelined commit + reduce on double-buffered replicas", 1, 0),
+                                 ("merge fused into the next local step", 0, 1)):
+            if (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
+                continue
+            setup(pipe, fuse, 1)
+            for t in range(3):
+                one_round(t)
+            hp.hpsgd_synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(main)
+            for t in range(args.other_schedule_steps):
+                one_round(3 + t)
+            hp.hpsgd_flush()
+            main.wait_stream(side)
+            b.record(main)
+            torch.cuda.synchronize(dev)
+            ms = a.elapsed_time(b) / args.other_schedule_steps
+            other[name] = {"ms_per_step": ms, "value": K * P / (ms * 1e-3), "steps": args.other_schedule_steps}
+        setup(args.pipeline, args.fuse, args.chunks)
+
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step
     e2e = None
     if args.e2e_steps > 0:
@@ -441,7 +469,7 @@ def run_gpu(args, cfg):
                 "l2": "inputs larger than L2 (state + gradients are tens of GB)",
                 "multi_gpu": "independent replicas, no inter-GPU exchange"}),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu,
+            "roofline": roofline, "cpu_baseline": cpu, "other_schedules": other,
         }
     hp.hpsgd_destroy()
     if dist is not None:
@@ -505,6 +533,8 @@ def main():
     ap.add_argument("--fuse", type=int, default=1, help="carry each merge into the next batched local step (one kernel)")
     ap.add_argument("--pipeline", type=int, default=0,
                     help="paper timeline: commit on the main stream, K-way reduce on the side stream, double-buffered replicas")
+    ap.add_argument("--other-schedule-steps", type=int, default=20,
+                    help="steps used to time each of the other schedules for the record (0 = skip)")
     ap.add_argument("--per-worker", action="store_true", help="K hpsgd_local_step calls instead of one batched call")
     ap.add_argument("--grad-buffers", type=int, default=2, help="rounds of device-resident gradients to cycle")
     ap.add_argument("--e2e-steps", type=int, default=3)
