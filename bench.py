@@ -395,7 +395,9 @@ def run_gpu(args, cfg):
     per_round = {"local_step_kernel": grad_bytes + state_bytes,
                  # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
                  "merge_kernel": (12 + (K + 2) * 4) * P if args.pipeline else merge_bytes_per_index(cfg) * P,
-                 "merge_step_kernel": 16 * P + grad_bytes + state_bytes}
+                 # fuse 2 with momentum: the replica rows are neither read nor written
+                 "merge_step_kernel": 16 * P + grad_bytes + (K * P * 8 if (args.fuse == 2 and cfg.momentum and K in (4, 8, 16))
+                                                             else state_bytes)}
     kernels = {}
     for name, (ms, n) in prof.items():
         if n == 0:
@@ -425,7 +427,8 @@ def run_gpu(args, cfg):
     if args.other_schedule_steps > 0 and not args.per_worker:
         for name, pipe, fuse in (("separate merge and local-step kernels on two streams", 0, 0),
                                  ("pipelined commit + reduce on double-buffered replicas", 1, 0),
-                                 ("merge fused into the next local step", 0, 1)):
+                                 ("merge fused into the next local step", 0, 1),
+                                 ("fused, replicas implicit (recomputed from momentum)", 0, 2)):
             if (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
                 continue
             setup(pipe, fuse, 1)
@@ -530,7 +533,9 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=workloads.names())
     ap.add_argument("--overlap", type=int, default=1)
     ap.add_argument("--chunks", type=int, default=1)
-    ap.add_argument("--fuse", type=int, default=1, help="carry each merge into the next batched local step (one kernel)")
+    ap.add_argument("--fuse", type=int, default=1,
+                    help="1: carry each merge into the next batched local step (one kernel); "
+                         "2: also leave the replicas implicit where fma(-mu, m, w) reproduces them; 0: separate kernels")
     ap.add_argument("--pipeline", type=int, default=0,
                     help="paper timeline: commit on the main stream, K-way reduce on the side stream, double-buffered replicas")
     ap.add_argument("--other-schedule-steps", type=int, default=20,

@@ -62,7 +62,13 @@ enum {
                                    both run as ONE kernel in which the re-cloned replica never goes
                                    to memory; any other call first launches the merge on its own.
                                    Same operations in the same order: results are bit-identical.
-                                   Default 0. */
+                                   2: as 1, and additionally, when momentum != 0, K is 4, 8 or 16 and
+                                   every worker made exactly one local step since the last merge, the
+                                   replica rows are neither read nor written: the replica the previous
+                                   step stored is fma(-mu, m_i, w) of values still in memory, and that
+                                   one FMA is recomputed instead (bit-identical).  The rows are rebuilt
+                                   before anything else reads them (hpsgd_synchronize, a per-worker
+                                   step, a merge on its own, a checkpoint).  Default 0. */
 };
 
 /* Kernel kinds of hpsgd_profile_read. */

@@ -96,6 +96,9 @@ struct Ctx {
     bool reduce_outstanding = false;
     bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
     int deferred_flags = 0;
+    std::vector<int> steps_in_period;      // local steps of each worker since the last merge request
+    bool deferred_all_single = false;      // every worker made exactly one step in the period the deferred merge closes
+    bool replicas_stale = false;           // replica rows not written by the implicit-replica kernel
     int64_t launches = 0;
     int sm_count = 148;
     int sp_tensor = -1;                    // sparse-row tensor
@@ -211,6 +214,23 @@ int prof_resolve()
     return HPSGD_OK;
 }
 
+// Rebuild replica rows that the implicit-replica kernel left stale: r_i = fma(-mu, m_i, w).
+int ensure_replicas()
+{
+    if (!g.replicas_stale) return HPSGD_OK;
+    const int64_t n = g.P_pad / 8;
+    dim3 grid(hot_grid(n), g.K);
+    materialize_kernel<<<grid, kHotThreads, 0, g.main>>>(g.w, g.m, g.r, g.stride, n, -g.lr);
+    ++g.launches;
+    g.replicas_stale = false;
+    if (g.overlap)
+        for (int c = 0; c < g.chunks; ++c) {
+            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
+            g.local_recorded[c] = 1;
+        }
+    return check_async();
+}
+
 // ---------------------------------------------------------------------------- local step
 struct LocalLaunch {
     int w0, nw;
@@ -261,6 +281,8 @@ void launch_accum_step(bool sparse, const LocalLaunch& L)
 // Enqueue the local step of workers [w0, w0 + nw) on the main stream, chunk by chunk.
 int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
 {
+    TRY(ensure_replicas());
+    for (int i = 0; i < nw; ++i) g.steps_in_period[w0 + i] += 1;
     LocalLaunch L{};
     L.w0 = w0; L.nw = nw; L.gp = gp;
     if (g.pipeline) {
@@ -382,6 +404,8 @@ int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; block
     CUDA_TRY(cudaStreamSynchronize(g.main));
     g.D_valid = false;
     g.merges = 0;
+    g.replicas_stale = false;
+    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 0);
     std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
     std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
     return HPSGD_OK;
@@ -471,6 +495,7 @@ void launch_accum_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
 // Enqueue one merge, chunk by chunk, on the side stream (main stream without overlap).
 int enqueue_merge(int flags)
 {
+    TRY(ensure_replicas());
     cudaStream_t s = g.overlap ? g.side : g.main;
     for (int c = 0; c < g.chunks; ++c) {
         int64_t lo, hi;
@@ -603,9 +628,35 @@ void launch_fused_k(bool mom, bool wd, bool sparse, const FusedLaunch& L)
     }
 }
 
+template <int KT>
+void launch_implicit(bool sparse, const FusedLaunch& L)
+{
+    const bool bf = g.grad_dtype == HPSGD_BF16, wd = g.lambda != 0.f;
+#define HPSGD_IMPLICIT_CASE(B, W, S)                                                                     \
+    merge_step_implicit_kernel<KT, B, W, S><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(                \
+        g.w, g.D, g.m, g.stride, L.gp, L.seg, L.o0, L.n, L.flags, L.p)
+    if (bf) {
+        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(true, true, true); else HPSGD_IMPLICIT_CASE(true, true, false); }
+        else { if (sparse) HPSGD_IMPLICIT_CASE(true, false, true); else HPSGD_IMPLICIT_CASE(true, false, false); }
+    } else {
+        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(false, true, true); else HPSGD_IMPLICIT_CASE(false, true, false); }
+        else { if (sparse) HPSGD_IMPLICIT_CASE(false, false, true); else HPSGD_IMPLICIT_CASE(false, false, false); }
+    }
+#undef HPSGD_IMPLICIT_CASE
+}
+
+// Can the deferred merge and the coming batched step run with the replicas left implicit?
+bool implicit_ok()
+{
+    return g.fuse == 2 && g.deferred_all_single && g.beta != 0.f && (g.K == 4 || g.K == 8 || g.K == 16);
+}
+
 // The deferred merge and the local step of all K workers in one kernel per chunk (main stream).
 int enqueue_fused(const BatchPtrs& gp, bool sparse)
 {
+    const bool implicit = implicit_ok();
+    if (!implicit) TRY(ensure_replicas());
+    for (int i = 0; i < g.K; ++i) g.steps_in_period[i] += 1;
     FusedLaunch L{};
     L.gp = gp;
     L.flags = g.deferred_flags;
@@ -629,7 +680,13 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
         L.o0 = lo; L.n = hi - lo;
         EventPair ep{};
         TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE_STEP, &ep));
-        if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
+        if (implicit) {
+            switch (g.K) {
+            case 4: launch_implicit<4>(sparse, L); break;
+            case 8: launch_implicit<8>(sparse, L); break;
+            default: launch_implicit<16>(sparse, L); break;
+            }
+        } else if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
         else launch_fused_k<false>(mom, wd, sparse, L);
         ++g.launches;
         TRY(prof_end(g.main, &ep));
@@ -638,6 +695,7 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
             g.local_recorded[c] = 1;
         }
     }
+    g.replicas_stale = implicit;
     return check_async();
 }
 
@@ -780,6 +838,7 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.r = reinterpret_cast<float*>(g.arena + a.r);
     g.m = mom ? reinterpret_cast<float*>(g.arena + a.m) : nullptr;
     g.d_table = reinterpret_cast<int64_t*>(g.arena + a.table);
+    g.steps_in_period.assign(K, 0);
     g.wbuf[0] = g.w;
     g.rbuf[0] = g.r;
     if (g.pipeline) {
@@ -844,6 +903,7 @@ int hpsgd_synchronize(void)
 {
     TRY(need_init());
     TRY(flush_deferred());
+    TRY(ensure_replicas());
     TRY(sync_all());
     return check_async();
 }
@@ -884,7 +944,7 @@ int hpsgd_set_option(int key, double value)
         TRY(sync_all());
         return make_chunk_events((int)value);
     case HPSGD_OPT_FUSE:
-        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "fuse must be 0 or 1");
+        if (value != 0.0 && value != 1.0 && value != 2.0) return fail(HPSGD_E_BADARG, "fuse must be 0, 1 or 2");
         g.fuse = (int)value;
         return HPSGD_OK;
     case HPSGD_OPT_PROFILE:
@@ -1038,6 +1098,12 @@ int hpsgd_sync_merge(void)
     else if (g.D_valid) flags |= kMergeApplyPending;
     g.D_valid = true;
     g.merges += 1;
+    bool all_single = true;
+    for (int& n : g.steps_in_period) {
+        all_single = all_single && n == 1;
+        n = 0;
+    }
+    g.deferred_all_single = all_single;
     if (g.pipeline) return enqueue_pipelined_merge(flags);
     if (g.fuse && g.form == HPSGD_FORM_REPLICA_CHANGE) {
         g.merge_deferred = true;
@@ -1134,6 +1200,7 @@ int hpsgd_export_state(void* host_out, size_t bytes)
     TRY(need_init());
     if (!host_out || bytes < state_bytes()) return fail(HPSGD_E_BADARG, "need a host buffer of hpsgd_state_bytes() = %zu bytes", state_bytes());
     TRY(flush_deferred());
+    TRY(ensure_replicas());
     TRY(sync_all());
     StateHeader h{};
     h.magic = kStateMagic;
@@ -1185,6 +1252,8 @@ int hpsgd_import_state(const void* host_in, size_t bytes)
     g.D_valid = h.D_valid != 0;
     g.merges = h.merges;
     if (g.pipeline) std::fill(g.touched.begin(), g.touched.end(), 1);   // every replica row now holds real data
+    g.replicas_stale = false;
+    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 2);   // unknown history: not "exactly one step"
     g.reduce_outstanding = false;
     std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
     std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);

@@ -608,6 +608,105 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
     }
 }
 
+// ---------------------------------------------------------------------------- merge + next local step, implicit replicas
+// With momentum and exactly one local step per worker since the last clone, the replica is
+// a function of state that is kept anyway: the step computed r_i = fma(-mu, m_i, w) from the
+// clone w and the new momentum m_i, both still in memory unchanged.  Recomputing that one FMA
+// gives the stored value bit for bit, so the replica rows need be neither read nor written:
+// per index the kernel moves (w + D + K m + K g) in and (w + D + K m) out, (3K + 4) * 4 bytes
+// with fp32 gradients instead of (5K + 4) * 4.  The replica rows are left stale;
+// materialize_kernel rebuilds them when something else needs them.
+template <int KT, bool BF16, bool WD, bool SPARSE>
+__global__ void __launch_bounds__(kHotThreads, 2)
+merge_step_implicit_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m,
+                           int64_t stride, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags,
+                           StepParams p)
+{
+    static_assert(KT > 0, "the momentum rows of all workers are held in registers");
+    constexpr int B = KT < 8 ? KT : 8;           // workers whose gradients are in flight together
+    const float fK = (float)KT;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        const int64_t e = o * 8;
+        SegPos sp{false, 0, 0};
+        int32_t sl[KT];
+        if (SPARSE) {
+            sp = seg_pos(seg, o);
+            if (sp.inside) {
+#pragma unroll
+                for (int i = 0; i < KT; ++i) sl[i] = __ldg(gp.slot[i] + sp.row);
+            }
+        }
+        const f8 wv = ld8(w + e);
+        f8 dv = zero8();
+        if (flags & kMergeApplyPending) dv = ld8(D + e);
+        f8 mv[KT];
+#pragma unroll
+        for (int i = 0; i < KT; ++i) mv[i] = ld8(m + (int64_t)i * stride + e);
+        // the gradients do not depend on the merge: the first batch is requested before it
+        GradRaw<BF16> graw[B];
+#pragma unroll
+        for (int b = 0; b < B; ++b) graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[b] : 0, b, o);
+        // ---- merge over the recomputed replicas r_i = w - mu*m_i
+        f8 acc;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(__fmaf_rn(p.neg_mu, mv[0].v[q], wv.v[q]), wv.v[q]);
+#pragma unroll
+        for (int i = 1; i < KT; ++i)
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(__fmaf_rn(p.neg_mu, mv[i].v[q], wv.v[q]), wv.v[q]));
+        f8 dnew, wn;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            dnew.v[q] = __fdiv_rn(acc.v[q], fK);
+            wn.v[q] = wv.v[q];
+            if (flags & kMergeImmediate) wn.v[q] = __fadd_rn(wv.v[q], dnew.v[q]);
+            else if (flags & kMergeApplyPending) wn.v[q] = __fadd_rn(wv.v[q], dv.v[q]);
+        }
+        st8(w + e, wn);
+        st8(D + e, dnew);
+        // ---- local step from the clone wn: only the momentum is stored
+#pragma unroll
+        for (int i0 = 0; i0 < KT; i0 += B) {
+            if (i0 > 0) {
+#pragma unroll
+                for (int b = 0; b < B; ++b)
+                    graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[i0 + b] : 0, i0 + b, o);
+            }
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                const f8 gg = widen_grad<BF16>(graw[b]);
+                f8 mn;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float gd = WD ? __fmaf_rn(p.lambda, wn.v[q], gg.v[q]) : gg.v[q];
+                    mn.v[q] = __fmaf_rn(p.beta, mv[i0 + b].v[q], gd);
+                }
+                st8(m + (int64_t)(i0 + b) * stride + e, mn);
+            }
+        }
+    }
+}
+
+// r_i = fma(-mu, m_i, w) for every worker (blockIdx.y): rebuilds replica rows left stale by
+// merge_step_implicit_kernel.
+__global__ void __launch_bounds__(kHotThreads)
+materialize_kernel(const float* __restrict__ w, const float* __restrict__ m, float* __restrict__ r,
+                   int64_t stride, int64_t n, float neg_mu)
+{
+    const int64_t off = (int64_t)blockIdx.y * stride;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
+        const f8 wv = ld8(w + o * 8);
+        const f8 mv = ld8(m + off + o * 8);
+        f8 rr;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) rr.v[q] = __fmaf_rn(neg_mu, mv.v[q], wv.v[q]);
+        st8(r + off + o * 8, rr);
+    }
+}
+
 // r_i = w for every worker (used when the state is (re)initialised).
 __global__ void __launch_bounds__(kThreads)
 clone_kernel(const float* __restrict__ w_, float* __restrict__ r_, int64_t stride, int K, int64_t nvec)

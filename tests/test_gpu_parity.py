@@ -384,11 +384,11 @@ def test_pipelined_sync_argument_checks():
 
 
 # ---------------------------------------------------------------- checkpoint
-@pytest.mark.parametrize("mode", ["plain", "fuse", "pipeline", "accum"])
+@pytest.mark.parametrize("mode", ["plain", "fuse", "implicit", "pipeline", "accum"])
 def test_export_import_resumes_bit_identically(mode):
     momentum = 0.0 if mode == "accum" else 0.9
     cfg = small("ckpt", 4, [20_000, 77], T=6, momentum=momentum, lr=0.05)
-    kw = dict(fuse=int(mode == "fuse"), pipeline=int(mode == "pipeline"),
+    kw = dict(fuse={"fuse": 1, "implicit": 2}.get(mode, 0), pipeline=int(mode == "pipeline"),
               form=hp.HPSGD_FORM_GRADIENT_ACCUMULATION if mode == "accum" else 0)
 
     def rounds(t0, t1, keep):
@@ -427,3 +427,54 @@ def test_more_workers_than_one_batched_launch_addresses():
     gu.run_both(cfg, cfg.T, batched=True)
     gu.run_both(cfg, cfg.T, batched=True, fuse=1, chunks=2)
     gu.run_both(cfg, cfg.T, batched=False)
+
+
+# ---------------------------------------------------------------- fused merge + step with implicit replicas
+@pytest.mark.parametrize("K,momentum,wd,staleness,H", [(16, 0.9, 0.0, 1, 1), (8, 0.9, 5e-4, 1, 1), (4, 0.5, 1e-3, 0, 1),
+                                                        (16, 0.9, 0.0, 1, 2), (3, 0.9, 0.0, 1, 1), (8, 0.0, 0.0, 1, 1)])
+def test_implicit_replicas_match_oracle(K, momentum, wd, staleness, H):
+    """HPSGD_OPT_FUSE = 2: replicas recomputed as fma(-mu, m, w) where that is exact; K = 3, plain SGD
+    and several steps per period take the ordinary fused path; all of it bit-identical."""
+    cfg = small("implicit", K, [70_001, 33, 4096], T=6, momentum=momentum, wd=wd, staleness=staleness)
+    gu.run_both(cfg, cfg.T, staleness=staleness, fuse=2, batched=True, chunks=2, steps_per_round=H)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_implicit_replicas_sparse_rows(dtype):
+    cfg = small("implicit_sparse", 4, [1000, 300 * 64, 777, 64], T=5, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
+    gu.run_both(cfg, cfg.T, fuse=2, batched=True)
+
+
+def test_implicit_replicas_are_rebuilt_on_demand():
+    """Interleave implicit rounds with calls that need real replica rows."""
+    cfg = small("implicit_mixed", 8, [40_000, 17], T=8, momentum=0.9, wd=1e-4)
+    o = gu.oracle_for(cfg)
+    with gu.session(cfg, fuse=2):
+        keep = []
+        launches = []
+        for t in range(cfg.T):
+            inputs = [gu.host_inputs(cfg, i, t) for i in range(cfg.K)]
+            for i, inp in enumerate(inputs):
+                o.local_step(i, inp["flat"])
+            if t == 4:                                   # per-worker calls in the middle of implicit rounds
+                for i, inp in enumerate(inputs):
+                    gu.gpu_step(cfg, i, inp, keep)
+            else:
+                stacked = np.stack([inp["padded"] for inp in inputs])
+                keep.append(gu.to_device(stacked.reshape(-1)))
+                before = hp.hpsgd_launch_count()
+                hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
+                launches.append(hp.hpsgd_launch_count() - before)
+            if t == 2:                                   # look at the replicas between step and merge
+                w, D, rs, ms = gu.gpu_state(cfg)
+                for i in range(cfg.K):
+                    gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d rebuilt from momentum" % i)
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+        assert launches[1] == 1 and launches[2] == 1     # one kernel per round while implicit
+        w, D, rs, ms = gu.gpu_state(cfg)
+        gu.assert_bitwise(w, o.get_global(), "global model")
+        gu.assert_bitwise(D, o.get_pending(), "pending change")
+        for i in range(cfg.K):
+            gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d" % i)
+            gu.assert_bitwise(ms[i], o.get_momentum(i), "momentum %d" % i)
