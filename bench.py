@@ -62,20 +62,24 @@ def fused_bytes_per_index(cfg):
 
 
 # DRAM bytes per parameter index (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture divided by the indices of that launch), keyed by (kernel, K, gradient dtype), with
+# capture divided by the indices of that launch), keyed by (kernel, K, gradient dtype, fuse variant), with
 # the SHA-1 of the kernel source the capture was taken from.  A changed source voids them.
 NCU_TRAFFIC = {
-    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200105 GB read + 2.123378 GB written over 16,000,000 indices
-    ("merge_step_kernel", 16, "f32"): {"bytes_per_index": 5.323483e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
-    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152239 GB + 1.093508 GB
-    ("merge_kernel", 16, "f32"): {"bytes_per_index": 2.245747e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
-    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072009 GB + 1.993030 GB (all 16 workers in one launch)
-    ("local_step_kernel", 16, "f32"): {"bytes_per_index": 5.065039e9 / 16e6, "source_sha1": "68dfc69bb09629a8df41874b140c72b24d1dc4f0"},
+    # profiles/merge_step_kernel_cfg4_cut16M.txt (second launch): 3.200035 GB read + 2.122386 GB written over 16,000,000 indices
+    ("merge_step_kernel", 16, "f32", 1): {"bytes_per_index": 5.322421e9 / 16e6, "source_sha1": "ed93d06b3a806d7be57c50338687b6f57d2ebd74"},
+    # profiles/merge_step_implicit_kernel_cfg4_cut16M.txt (second launch): 2.176028 GB + 1.124347 GB
+    ("merge_step_kernel", 16, "f32", 2): {"bytes_per_index": 3.300375e9 / 16e6, "source_sha1": "ed93d06b3a806d7be57c50338687b6f57d2ebd74"},
+    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152057 GB + 1.096189 GB
+    ("merge_kernel", 16, "f32", 0): {"bytes_per_index": 2.248246e9 / 16e6, "source_sha1": "ed93d06b3a806d7be57c50338687b6f57d2ebd74"},
+    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072010 GB + 1.997191 GB (all 16 workers in one launch)
+    ("local_step_kernel", 16, "f32", 0): {"bytes_per_index": 5.069201e9 / 16e6, "source_sha1": "ed93d06b3a806d7be57c50338687b6f57d2ebd74"},
 }
 
 
-def ncu_traffic(kernel, cfg, algorithmic_bytes_per_launch):
-    entry = NCU_TRAFFIC.get((kernel, cfg.K, cfg.grad_dtype))
+def ncu_traffic(kernel, cfg, fuse):
+    """Measured DRAM bytes of one full launch of that kernel on this workload, or None."""
+    variant = fuse if kernel == "merge_step_kernel" else 0
+    entry = NCU_TRAFFIC.get((kernel, cfg.K, cfg.grad_dtype, variant))
     if entry is None:
         return None
     import hashlib
@@ -411,7 +415,7 @@ def run_gpu(args, cfg):
     dominant = max(kernels, key=lambda k: kernels[k]["total_ms"])
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved"], "peak": peak,
                 "unit": "GB/s", "frac": kernels[dominant]["frac"],
-                "traffic": ncu_traffic(dominant, cfg, kernels[dominant]["algorithmic_bytes_per_launch"]),
+                "traffic": ncu_traffic(dominant, cfg, args.fuse) if (args.chunks == 1 and not args.per_worker) else None,
                 "peak_source": peak_src, "nominal_peak": NOMINAL_HBM_GBS, "kernels": kernels,
                 "note": "CUDA event pairs around each launch on its own stream inside the timed region; "
                         "a fused merge_step_kernel launch moves 16 + K*(local step bytes) per index, "
