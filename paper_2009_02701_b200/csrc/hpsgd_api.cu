@@ -1,705 +1,7 @@
-// C ABI of libhpsgd: state, validation, stream/event schedule and kernel launches.
-// The contract of every entry point is documented in include/hpsgd.h.
-#include "../../include/hpsgd.h"
-
-#include <algorithm>
-#include <cstdarg>
-#include <cstdio>
-#include <cstring>
-#include <vector>
-
-#include "hpsgd_kernels.cuh"
-
-namespace {
-
-using namespace hpsgd;
-
-constexpr int64_t kAlignElems = 32;        // tensor starts: multiples of 32 elements
-constexpr int64_t kRowAlignElems = 64;     // rows of r / m: multiples of 256 bytes
-constexpr size_t kAlignBytes = 256;        // arena regions
-constexpr int kMaxChunks = 1024;
-constexpr int kMaxTensors = 4096;
-constexpr int64_t kChunkGrain = 1024;      // chunk boundaries: multiples of 1024 groups (8192 elements)
-constexpr int kMaxGridX = 0x7FFFFFFF;
-
-char g_err[512] = "";
-
-int fail(int code, const char* fmt, ...)
-{
-    va_list ap;
-    va_start(ap, fmt);
-    vsnprintf(g_err, sizeof g_err, fmt, ap);
-    va_end(ap);
-    return code;
-}
-
-#define CUDA_TRY(expr)                                                                      \
-    do {                                                                                    \
-        cudaError_t e_ = (expr);                                                            \
-        if (e_ != cudaSuccess)                                                              \
-            return fail(HPSGD_E_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));      \
-    } while (0)
-
-#define TRY(expr)                \
-    do {                         \
-        int rc_ = (expr);        \
-        if (rc_) return rc_;     \
-    } while (0)
-
-size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-struct EventPair {
-    cudaEvent_t a, b;
-    int kind;       // HPSGD_KERNEL_*
-};
-
-struct Pending {                // configuration collected before hpsgd_init
-    std::vector<int64_t> sizes;
-    void* arena = nullptr;
-    size_t arena_bytes = 0;
-    cudaStream_t main = nullptr, side = nullptr;
-    bool have_streams = false;
-    int form = HPSGD_FORM_REPLICA_CHANGE;
-    int pipeline = 0;
-} g_pending;
-
-struct Ctx {
-    bool inited = false;
-    int64_t P = 0, P_pad = 0, stride = 0;  // stride: floats between consecutive workers' rows
-    int K = 0;
-    float lr = 0.f, beta = 0.f, lambda = 0.f;
-    uint64_t seed = 0, key = 0;
-    int staleness = 1, grad_dtype = HPSGD_F32, overlap = 1, chunks = 1, profile = 0;
-    std::vector<int64_t> sizes, offsets, starts;
-    int64_t* d_table = nullptr;            // offsets | starts | sizes, on the device
-    char* arena = nullptr;
-    size_t arena_bytes = 0;
-    bool own_arena = false;
-    float *w = nullptr, *D = nullptr, *r = nullptr, *m = nullptr;
-    int32_t* slot = nullptr;               // [K][slot_cap] row -> slot scratch map
-    int64_t slot_cap = 0;
-    bool own_slot = false;
-    cudaStream_t main = nullptr, side = nullptr, copy = nullptr;
-    bool own_streams = false;
-    std::vector<cudaEvent_t> ev_local, ev_merge;
-    std::vector<char> local_recorded, merge_unwaited;
-    bool D_valid = false;
-    int64_t merges = 0;
-    int form = HPSGD_FORM_REPLICA_CHANGE;  // what the workers carry: replica change or accumulated gradients
-    int fuse = 0;                          // carry a merge into the next batched local step
-    int pipeline = 0;                      // commit/reduce split on double-buffered replicas
-    float* wbuf[2] = {nullptr, nullptr};   // pipeline: global model of the current / other period
-    float* rbuf[2] = {nullptr, nullptr};   // pipeline: replica sets of the current / other period
-    int cur = 0;                           // pipeline: which buffers the current period trains on
-    std::vector<char> touched;             // pipeline: worker has made a local step this period
-    cudaEvent_t ev_commit = nullptr, ev_reduce = nullptr;
-    bool reduce_outstanding = false;
-    bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
-    int deferred_flags = 0;
-    std::vector<int> steps_in_period;      // local steps of each worker since the last merge request
-    bool deferred_all_single = false;      // every worker made exactly one step in the period the deferred merge closes
-    bool replicas_stale = false;           // replica rows not written by the implicit-replica kernel
-    int64_t launches = 0;
-    int sm_count = 148;
-    int sp_tensor = -1;                    // sparse-row tensor
-    int64_t sp_rows = 0, sp_cols = 0;
-    void* stage[2] = {nullptr, nullptr};   // staging of hpsgd_local_step_host
-    cudaEvent_t stage_copied[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
-    bool stage_used[2] = {false, false};
-    int stage_next = 0;
-    std::vector<EventPair> prof;           // profiling
-    double prof_ms[3] = {0, 0, 0};
-    int64_t prof_launches[3] = {0, 0, 0};
-} g;
-
-int check_async()
-{
-    cudaError_t e = cudaPeekAtLastError();
-    if (e != cudaSuccess) return fail(HPSGD_E_CUDA, "CUDA error: %s", cudaGetErrorString(e));
-    return HPSGD_OK;
-}
-
-int64_t layout_of(const std::vector<int64_t>& sizes, std::vector<int64_t>* offsets, std::vector<int64_t>* starts)
-{
-    int64_t pos = 0, flat = 0;
-    for (int64_t s : sizes) {
-        if (offsets) offsets->push_back(pos);
-        if (starts) starts->push_back(flat);
-        pos += (s + kAlignElems - 1) / kAlignElems * kAlignElems;
-        flat += s;
-    }
-    return pos;
-}
-
-// Regions of the arena, in order: w | D | r[K] | m[K] | w2 | r2[K] | table | slot maps (the rest).
-struct ArenaPlan {
-    size_t w, D, r, m, w2, r2, table, slot, fixed;
-};
-
-ArenaPlan plan_arena(int64_t stride, int K, bool momentum, bool pipeline)
-{
-    ArenaPlan a{};
-    const size_t row = (size_t)stride * 4;
-    size_t pos = 0;
-    a.w = pos; pos += row;
-    a.D = pos; pos += row;
-    a.r = pos; pos += row * K;
-    a.m = pos; if (momentum) pos += row * K;
-    a.w2 = pos; if (pipeline) pos += row;
-    a.r2 = pos; if (pipeline) pos += row * K;
-    a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kAlignBytes);
-    a.slot = pos;
-    a.fixed = pos;
-    return a;
-}
-
-// Index range [o_lo, o_hi), in 8-element groups, of schedule chunk c.
-void chunk_range(int c, int64_t* o_lo, int64_t* o_hi)
-{
-    const int64_t n = g.P_pad / 8;
-    const int64_t grains = (n + kChunkGrain - 1) / kChunkGrain;
-    auto edge = [&](int k) { return std::min(n, grains * k / g.chunks * kChunkGrain); };
-    *o_lo = edge(c);
-    *o_hi = (c == g.chunks - 1) ? n : edge(c + 1);
-}
-
-// Grid of the hot kernels: one block per kHotThreads groups.
-int hot_grid(int64_t groups)
-{
-    return (int)std::min<int64_t>(kMaxGridX, std::max<int64_t>(1, (groups + kHotThreads - 1) / kHotThreads));
-}
-
-// Grid of the support kernels: enough blocks to cover `items`, capped at one full wave of
-// resident blocks (SM count x blocks the kernel can keep resident per SM).
-template <typename Kern>
-int grid_for(Kern kern, int64_t items, int64_t per_block)
-{
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0) != cudaSuccess || occ < 1) occ = 1;
-    const int64_t need = std::max<int64_t>(1, (items + per_block - 1) / per_block);
-    return (int)std::min<int64_t>(need, (int64_t)g.sm_count * occ);
-}
-
-// ---------------------------------------------------------------------------- profiling
-int prof_begin(cudaStream_t s, int kind, EventPair* ep)
-{
-    if (!g.profile) return HPSGD_OK;
-    ep->kind = kind;
-    CUDA_TRY(cudaEventCreate(&ep->a));
-    CUDA_TRY(cudaEventCreate(&ep->b));
-    CUDA_TRY(cudaEventRecord(ep->a, s));
-    return HPSGD_OK;
-}
-
-int prof_end(cudaStream_t s, EventPair* ep)
-{
-    if (!g.profile) return HPSGD_OK;
-    CUDA_TRY(cudaEventRecord(ep->b, s));
-    g.prof.push_back(*ep);
-    return HPSGD_OK;
-}
-
-int prof_resolve()
-{
-    for (EventPair& ep : g.prof) {
-        CUDA_TRY(cudaEventSynchronize(ep.b));
-        float ms = 0.f;
-        CUDA_TRY(cudaEventElapsedTime(&ms, ep.a, ep.b));
-        g.prof_ms[ep.kind] += ms;
-        g.prof_launches[ep.kind] += 1;
-        cudaEventDestroy(ep.a);
-        cudaEventDestroy(ep.b);
-    }
-    g.prof.clear();
-    return HPSGD_OK;
-}
-
-// Rebuild replica rows that the implicit-replica kernel left stale: r_i = fma(-mu, m_i, w).
-int ensure_replicas()
-{
-    if (!g.replicas_stale) return HPSGD_OK;
-    const int64_t n = g.P_pad / 8;
-    dim3 grid(hot_grid(n), g.K);
-    materialize_kernel<<<grid, kHotThreads, 0, g.main>>>(g.w, g.m, g.r, g.stride, n, -g.lr);
-    ++g.launches;
-    g.replicas_stale = false;
-    if (g.overlap)
-        for (int c = 0; c < g.chunks; ++c) {
-            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
-            g.local_recorded[c] = 1;
-        }
-    return check_async();
-}
-
-// ---------------------------------------------------------------------------- local step
-struct LocalLaunch {
-    int w0, nw;
-    BatchPtrs gp;
-    SparseSeg seg;
-    int64_t o0, n;
-    StepParams p;
-};
-
-template <bool BF16, bool MOM, bool WD, bool SPARSE>
-void launch_local(const LocalLaunch& L)
-{
-    dim3 grid(hot_grid(L.n), L.nw);
-    local_step_kernel<BF16, MOM, WD, SPARSE><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp,
-                                                                               L.seg, L.o0, L.n, L.p);
-}
-
-template <bool BF16, bool MOM, bool WD>
-void launch_local_s(bool sparse, const LocalLaunch& L)
-{
-    if (sparse) launch_local<BF16, MOM, WD, true>(L);
-    else launch_local<BF16, MOM, WD, false>(L);
-}
-
-template <bool BF16>
-void launch_local_d(bool mom, bool wd, bool sparse, const LocalLaunch& L)
-{
-    if (mom && wd) launch_local_s<BF16, true, true>(sparse, L);
-    else if (mom) launch_local_s<BF16, true, false>(sparse, L);
-    else if (wd) launch_local_s<BF16, false, true>(sparse, L);
-    else launch_local_s<BF16, false, false>(sparse, L);
-}
-
-// Gradient-accumulation form: r -= mu*g, a += g (the accumulators live where momentum would).
-void launch_accum_step(bool sparse, const LocalLaunch& L)
-{
-    dim3 grid(hot_grid(L.n), L.nw);
-    const bool bf = g.grad_dtype == HPSGD_BF16;
-#define HPSGD_ACCUM_CASE(B, S) \
-    accum_step_kernel<B, S><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.o0, L.n, L.p.neg_mu)
-    if (bf && sparse) HPSGD_ACCUM_CASE(true, true);
-    else if (bf) HPSGD_ACCUM_CASE(true, false);
-    else if (sparse) HPSGD_ACCUM_CASE(false, true);
-    else HPSGD_ACCUM_CASE(false, false);
-#undef HPSGD_ACCUM_CASE
-}
-
-// Enqueue the local step of workers [w0, w0 + nw) on the main stream, chunk by chunk.
-int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
-{
-    TRY(ensure_replicas());
-    for (int i = 0; i < nw; ++i) g.steps_in_period[w0 + i] += 1;
-    LocalLaunch L{};
-    L.w0 = w0; L.nw = nw; L.gp = gp;
-    if (g.pipeline) {
-        // first step of a worker in this period: its replica is still the clone, i.e. w itself
-        for (int i = 0; i < nw; ++i) {
-            if (!g.touched[w0 + i]) {
-                L.gp.r_src[i] = g.w;
-                g.touched[w0 + i] = 1;
-            }
-        }
-    }
-    L.p = StepParams{-g.lr, g.beta, g.lambda};
-    L.seg = SparseSeg{0, 0, 1};
-    if (sparse) {
-        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
-        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
-        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
-    }
-    const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
-    for (int c = 0; c < g.chunks; ++c) {
-        int64_t lo, hi;
-        chunk_range(c, &lo, &hi);
-        if (hi <= lo) continue;
-        if (g.merge_unwaited[c]) {
-            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
-            g.merge_unwaited[c] = 0;
-        }
-        L.o0 = lo; L.n = hi - lo;
-        EventPair ep{};
-        TRY(prof_begin(g.main, HPSGD_KERNEL_LOCAL_STEP, &ep));
-        if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) launch_accum_step(sparse, L);
-        else if (g.grad_dtype == HPSGD_BF16) launch_local_d<true>(mom, wd, sparse, L);
-        else launch_local_d<false>(mom, wd, sparse, L);
-        ++g.launches;
-        TRY(prof_end(g.main, &ep));
-        if (g.overlap) {
-            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
-            g.local_recorded[c] = 1;
-        }
-    }
-    return check_async();
-}
-
-// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors: one memset over
-// the nw consecutive maps (every row: no slot, -1) and one scatter launch for all of them.
-int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* gp)
-{
-    int32_t* first = g.slot + (int64_t)w0 * g.slot_cap;
-    CUDA_TRY(cudaMemsetAsync(first, 0xFF, (size_t)g.slot_cap * 4 * nw, g.main));
-    SlotBatch sb{};
-    int32_t most = 0;
-    for (int i = 0; i < nw; ++i) {
-        const hpsgd_grad_desc& d = descs[i];
-        sb.slot[i] = first + (int64_t)i * g.slot_cap;
-        sb.row_idx[i] = d.row_idx;
-        sb.n_rows[i] = (d.row_idx && d.n_rows > 0) ? d.n_rows : 0;
-        most = std::max(most, sb.n_rows[i]);
-        gp->slot[i] = sb.slot[i];
-        gp->row_vals[i] = d.row_vals;
-        gp->dense[i] = d.dense;
-    }
-    if (most > 0) {
-        scatter_slots_kernel<<<dim3((most + 255) / 256, nw), 256, 0, g.main>>>(sb, g.sp_rows);
-        ++g.launches;
-    }
-    return HPSGD_OK;
-}
-
-int check_grad_ptr(const void* p, const char* what)
-{
-    if (!p) return fail(HPSGD_E_BADARG, "%s is NULL", what);
-    if (reinterpret_cast<uintptr_t>(p) % 32) return fail(HPSGD_E_BADARG, "%s is not 32-byte aligned", what);
-    return HPSGD_OK;
-}
-
-int check_desc(const hpsgd_grad_desc* d)
-{
-    if (!d) return fail(HPSGD_E_BADARG, "descriptor is NULL");
-    TRY(check_grad_ptr(d->dense, "dense gradient"));
-    if (d->n_rows < 0 || d->n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows %d out of range", d->n_rows);
-    if (d->n_rows > 0 && d->row_idx) TRY(check_grad_ptr(d->row_vals, "row_vals"));
-    return HPSGD_OK;
-}
-
-int need_init()
-{
-    if (!g.inited) return fail(HPSGD_E_STATE, "hpsgd_init has not been called");
-    return HPSGD_OK;
-}
-
-int check_worker(int worker)
-{
-    if (worker < 0 || worker >= g.K) return fail(HPSGD_E_BADARG, "worker %d outside [0, %d)", worker, g.K);
-    return HPSGD_OK;
-}
-
-int sync_all()
-{
-    CUDA_TRY(cudaStreamSynchronize(g.main));
-    CUDA_TRY(cudaStreamSynchronize(g.side));
-    if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
-    return HPSGD_OK;
-}
-
-int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; blocking
-{
-    const size_t row = (size_t)g.stride * 4;
-    CUDA_TRY(cudaMemsetAsync(g.D, 0, row, g.main));
-    if (g.m) CUDA_TRY(cudaMemsetAsync(g.m, 0, row * g.K, g.main));
-    if (g.pipeline) {
-        std::fill(g.touched.begin(), g.touched.end(), 0);      // replicas are w until their first step
-        g.reduce_outstanding = false;
-    } else {
-        const int64_t nvec = g.P_pad / 4;
-        clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
-        ++g.launches;
-        CUDA_TRY(cudaGetLastError());
-    }
-    CUDA_TRY(cudaStreamSynchronize(g.main));
-    g.D_valid = false;
-    g.merges = 0;
-    g.replicas_stale = false;
-    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 0);
-    std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
-    std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
-    return HPSGD_OK;
-}
-
-int make_chunk_events(int chunks)
-{
-    for (cudaEvent_t e : g.ev_local) cudaEventDestroy(e);
-    for (cudaEvent_t e : g.ev_merge) cudaEventDestroy(e);
-    g.ev_local.assign(chunks, nullptr);
-    g.ev_merge.assign(chunks, nullptr);
-    g.local_recorded.assign(chunks, 0);
-    g.merge_unwaited.assign(chunks, 0);
-    g.chunks = chunks;
-    for (int c = 0; c < chunks; ++c) {
-        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_local[c], cudaEventDisableTiming));
-        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_merge[c], cudaEventDisableTiming));
-    }
-    return HPSGD_OK;
-}
-
-GenParams gen_params(int worker, int step, int kind, double scale)
-{
-    GenParams gp{};
-    gp.key = g.key;
-    gp.step = (uint64_t)step;
-    gp.worker = (uint64_t)worker;
-    gp.kind = kind;
-    gp.scale_f = (float)scale;
-    gp.scale_d = scale;
-    if (g.sp_tensor >= 0) {
-        gp.sp_start = g.starts[g.sp_tensor];
-        gp.sp_rows = g.sp_rows;
-        gp.sp_cols = g.sp_cols;
-    }
-    return gp;
-}
-
-int check_gen_args(const void* out, int worker, int step, int kind)
-{
-    TRY(need_init());
-    TRY(check_grad_ptr(out, "output buffer"));
-    if (worker < 0 || worker >= 256) return fail(HPSGD_E_BADARG, "worker must be in [0, 256)");
-    if (step < 0 || step >= (1 << 20)) return fail(HPSGD_E_BADARG, "step must be in [0, 2^20)");
-    if (kind != HPSGD_GEN_UNIFORM && kind != HPSGD_GEN_GAUSS) return fail(HPSGD_E_BADARG, "unknown generator kind");
-    return HPSGD_OK;
-}
-
-void release_all()
-{
-    if (g.main) cudaStreamSynchronize(g.main);
-    if (g.side) cudaStreamSynchronize(g.side);
-    if (g.copy) cudaStreamSynchronize(g.copy);
-    for (EventPair& ep : g.prof) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
-    for (cudaEvent_t e : g.ev_local) if (e) cudaEventDestroy(e);
-    for (cudaEvent_t e : g.ev_merge) if (e) cudaEventDestroy(e);
-    if (g.ev_commit) cudaEventDestroy(g.ev_commit);
-    if (g.ev_reduce) cudaEventDestroy(g.ev_reduce);
-    for (int b = 0; b < 2; ++b) {
-        if (g.stage[b]) cudaFree(g.stage[b]);
-        if (g.stage_copied[b]) cudaEventDestroy(g.stage_copied[b]);
-        if (g.stage_free[b]) cudaEventDestroy(g.stage_free[b]);
-    }
-    if (g.copy) cudaStreamDestroy(g.copy);
-    if (g.own_streams) {
-        if (g.main) cudaStreamDestroy(g.main);
-        if (g.side) cudaStreamDestroy(g.side);
-    }
-    if (g.own_slot && g.slot) cudaFree(g.slot);
-    if (g.own_arena && g.arena) cudaFree(g.arena);
-    cudaGetLastError();
-    g = Ctx();
-}
-
-template <int KT>
-void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
-{
-    merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags);
-}
-
-template <int KT>
-void launch_accum_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
-{
-    accum_merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.m, g.stride, g.K, o0, n, flags, -g.lr);
-}
-
-// Enqueue one merge, chunk by chunk, on the side stream (main stream without overlap).
-int enqueue_merge(int flags)
-{
-    TRY(ensure_replicas());
-    cudaStream_t s = g.overlap ? g.side : g.main;
-    for (int c = 0; c < g.chunks; ++c) {
-        int64_t lo, hi;
-        chunk_range(c, &lo, &hi);
-        if (hi <= lo) continue;
-        if (g.overlap && g.local_recorded[c]) {
-            CUDA_TRY(cudaStreamWaitEvent(s, g.ev_local[c], 0));
-            g.local_recorded[c] = 0;
-        }
-        EventPair ep{};
-        TRY(prof_begin(s, HPSGD_KERNEL_MERGE, &ep));
-        if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) {
-            switch (g.K) {
-            case 4: launch_accum_merge<4>(s, lo, hi - lo, flags); break;
-            case 8: launch_accum_merge<8>(s, lo, hi - lo, flags); break;
-            case 16: launch_accum_merge<16>(s, lo, hi - lo, flags); break;
-            default: launch_accum_merge<0>(s, lo, hi - lo, flags); break;
-            }
-        } else {
-            switch (g.K) {
-            case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
-            case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
-            case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
-            default: launch_merge<0>(s, lo, hi - lo, flags); break;
-            }
-        }
-        ++g.launches;
-        TRY(prof_end(s, &ep));
-        if (g.overlap) {
-            CUDA_TRY(cudaEventRecord(g.ev_merge[c], s));
-            g.merge_unwaited[c] = 1;
-        }
-    }
-    return check_async();
-}
-
-template <int KT>
-void launch_reduce(const float* w_old, const ReducePtrs& rp, int64_t n)
-{
-    reduce_kernel<KT><<<hot_grid(n), kHotThreads, 0, g.side>>>(w_old, g.D, rp, g.K, n);
-}
-
-// Pipelined synchronisation: the commit w_next = w + D runs on the main stream, in order with
-// the local steps; the K-way reduce of the period that just ended runs on the side stream and
-// nothing on the main stream waits for it until the NEXT synchronisation needs its result.
-int enqueue_pipelined_merge(int flags)
-{
-    const int64_t n = g.P_pad / 8;
-    const int nxt = g.cur ^ 1;
-    if (g.reduce_outstanding) {
-        // the previous reduce still reads the buffers about to be written and produces the D read here
-        CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_reduce, 0));
-        g.reduce_outstanding = false;
-    }
-    EventPair ep{};
-    TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE, &ep));
-    commit_kernel<<<hot_grid(n), kHotThreads, 0, g.main>>>(g.wbuf[g.cur], g.D, g.wbuf[nxt], n, flags);
-    ++g.launches;
-    TRY(prof_end(g.main, &ep));
-    CUDA_TRY(cudaEventRecord(g.ev_commit, g.main));
-    CUDA_TRY(cudaStreamWaitEvent(g.side, g.ev_commit, 0));
-    ReducePtrs rp{};
-    for (int i = 0; i < g.K; ++i)
-        rp.src[i] = g.touched[i] ? g.rbuf[g.cur] + (int64_t)i * g.stride : g.wbuf[g.cur];
-    EventPair ep2{};
-    TRY(prof_begin(g.side, HPSGD_KERNEL_MERGE, &ep2));
-    switch (g.K) {
-    case 4: launch_reduce<4>(g.wbuf[g.cur], rp, n); break;
-    case 8: launch_reduce<8>(g.wbuf[g.cur], rp, n); break;
-    case 16: launch_reduce<16>(g.wbuf[g.cur], rp, n); break;
-    default: launch_reduce<0>(g.wbuf[g.cur], rp, n); break;
-    }
-    ++g.launches;
-    TRY(prof_end(g.side, &ep2));
-    CUDA_TRY(cudaEventRecord(g.ev_reduce, g.side));
-    g.reduce_outstanding = true;
-    g.cur = nxt;
-    g.w = g.wbuf[nxt];
-    g.r = g.rbuf[nxt];
-    std::fill(g.touched.begin(), g.touched.end(), 0);
-    return check_async();
-}
-
-// A merge that hpsgd_sync_merge deferred (fuse option) and that nothing has absorbed yet.
-int flush_deferred()
-{
-    if (!g.merge_deferred) return HPSGD_OK;
-    g.merge_deferred = false;
-    return enqueue_merge(g.deferred_flags);
-}
-
-struct FusedLaunch {
-    BatchPtrs gp;
-    SparseSeg seg;
-    int64_t o0, n;
-    int flags;
-    StepParams p;
-};
-
-template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
-void launch_fused(const FusedLaunch& L)
-{
-    merge_step_kernel<KT, BF16, MOM, WD, SPARSE><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
-        g.w, g.D, g.r, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p);
-}
-
-template <int KT, bool BF16>
-void launch_fused_d(bool mom, bool wd, bool sparse, const FusedLaunch& L)
-{
-#define HPSGD_FUSED_CASE(M, W)                                    \
-    do {                                                          \
-        if (sparse) launch_fused<KT, BF16, M, W, true>(L);        \
-        else launch_fused<KT, BF16, M, W, false>(L);              \
-    } while (0)
-    if (mom && wd) HPSGD_FUSED_CASE(true, true);
-    else if (mom) HPSGD_FUSED_CASE(true, false);
-    else if (wd) HPSGD_FUSED_CASE(false, true);
-    else HPSGD_FUSED_CASE(false, false);
-#undef HPSGD_FUSED_CASE
-}
-
-template <bool BF16>
-void launch_fused_k(bool mom, bool wd, bool sparse, const FusedLaunch& L)
-{
-    switch (g.K) {
-    case 4: launch_fused_d<4, BF16>(mom, wd, sparse, L); break;
-    case 8: launch_fused_d<8, BF16>(mom, wd, sparse, L); break;
-    case 16: launch_fused_d<16, BF16>(mom, wd, sparse, L); break;
-    default: launch_fused_d<0, BF16>(mom, wd, sparse, L); break;
-    }
-}
-
-template <int KT>
-void launch_implicit(bool sparse, const FusedLaunch& L)
-{
-    const bool bf = g.grad_dtype == HPSGD_BF16, wd = g.lambda != 0.f;
-#define HPSGD_IMPLICIT_CASE(B, W, S)                                                                     \
-    merge_step_implicit_kernel<KT, B, W, S><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(                \
-        g.w, g.D, g.m, g.stride, L.gp, L.seg, L.o0, L.n, L.flags, L.p)
-    if (bf) {
-        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(true, true, true); else HPSGD_IMPLICIT_CASE(true, true, false); }
-        else { if (sparse) HPSGD_IMPLICIT_CASE(true, false, true); else HPSGD_IMPLICIT_CASE(true, false, false); }
-    } else {
-        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(false, true, true); else HPSGD_IMPLICIT_CASE(false, true, false); }
-        else { if (sparse) HPSGD_IMPLICIT_CASE(false, false, true); else HPSGD_IMPLICIT_CASE(false, false, false); }
-    }
-#undef HPSGD_IMPLICIT_CASE
-}
-
-// Can the deferred merge and the coming batched step run with the replicas left implicit?
-bool implicit_ok()
-{
-    return g.fuse == 2 && g.deferred_all_single && g.beta != 0.f && (g.K == 4 || g.K == 8 || g.K == 16);
-}
-
-// The deferred merge and the local step of all K workers in one kernel per chunk (main stream).
-int enqueue_fused(const BatchPtrs& gp, bool sparse)
-{
-    const bool implicit = implicit_ok();
-    if (!implicit) TRY(ensure_replicas());
-    for (int i = 0; i < g.K; ++i) g.steps_in_period[i] += 1;
-    FusedLaunch L{};
-    L.gp = gp;
-    L.flags = g.deferred_flags;
-    L.p = StepParams{-g.lr, g.beta, g.lambda};
-    L.seg = SparseSeg{0, 0, 1};
-    if (sparse) {
-        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
-        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
-        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
-    }
-    g.merge_deferred = false;
-    const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
-    for (int c = 0; c < g.chunks; ++c) {
-        int64_t lo, hi;
-        chunk_range(c, &lo, &hi);
-        if (hi <= lo) continue;
-        if (g.merge_unwaited[c]) {
-            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
-            g.merge_unwaited[c] = 0;
-        }
-        L.o0 = lo; L.n = hi - lo;
-        EventPair ep{};
-        TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE_STEP, &ep));
-        if (implicit) {
-            switch (g.K) {
-            case 4: launch_implicit<4>(sparse, L); break;
-            case 8: launch_implicit<8>(sparse, L); break;
-            default: launch_implicit<16>(sparse, L); break;
-            }
-        } else if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
-        else launch_fused_k<false>(mom, wd, sparse, L);
-        ++g.launches;
-        TRY(prof_end(g.main, &ep));
-        if (g.overlap) {
-            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
-            g.local_recorded[c] = 1;
-        }
-    }
-    g.replicas_stale = implicit;
-    return check_async();
-}
-
-}  // namespace
+// C ABI of libhpsgd: the entry points.  The contract of every entry point is documented in
+// include/hpsgd.h; state and helpers live in hpsgd_state.cuh, the stream/event schedule and the
+// kernel launches in hpsgd_schedule.cuh, the device code in hpsgd_kernels.cuh.
+#include "hpsgd_schedule.cuh"
 
 // =============================================================================== C ABI
 extern "C" {

@@ -1,0 +1,349 @@
+// Internal state of libhpsgd: the singleton context, arena plan, index ranges of the
+// schedule, grids, profiling events and the small helpers every entry point uses.
+// Included by hpsgd_api.cu only (one translation unit).
+#pragma once
+
+#include "../../include/hpsgd.h"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "hpsgd_kernels.cuh"
+
+namespace {
+
+using namespace hpsgd;
+
+constexpr int64_t kAlignElems = 32;        // tensor starts: multiples of 32 elements
+constexpr int64_t kRowAlignElems = 64;     // rows of r / m: multiples of 256 bytes
+constexpr size_t kAlignBytes = 256;        // arena regions
+constexpr int kMaxChunks = 1024;
+constexpr int kMaxTensors = 4096;
+constexpr int64_t kChunkGrain = 1024;      // chunk boundaries: multiples of 1024 groups (8192 elements)
+constexpr int kMaxGridX = 0x7FFFFFFF;
+
+char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                      \
+    do {                                                                                    \
+        cudaError_t e_ = (expr);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return fail(HPSGD_E_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));      \
+    } while (0)
+
+#define TRY(expr)                \
+    do {                         \
+        int rc_ = (expr);        \
+        if (rc_) return rc_;     \
+    } while (0)
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct EventPair {
+    cudaEvent_t a, b;
+    int kind;       // HPSGD_KERNEL_*
+};
+
+struct Pending {                // configuration collected before hpsgd_init
+    std::vector<int64_t> sizes;
+    void* arena = nullptr;
+    size_t arena_bytes = 0;
+    cudaStream_t main = nullptr, side = nullptr;
+    bool have_streams = false;
+    int form = HPSGD_FORM_REPLICA_CHANGE;
+    int pipeline = 0;
+} g_pending;
+
+struct Ctx {
+    bool inited = false;
+    int64_t P = 0, P_pad = 0, stride = 0;  // stride: floats between consecutive workers' rows
+    int K = 0;
+    float lr = 0.f, beta = 0.f, lambda = 0.f;
+    uint64_t seed = 0, key = 0;
+    int staleness = 1, grad_dtype = HPSGD_F32, overlap = 1, chunks = 1, profile = 0;
+    std::vector<int64_t> sizes, offsets, starts;
+    int64_t* d_table = nullptr;            // offsets | starts | sizes, on the device
+    char* arena = nullptr;
+    size_t arena_bytes = 0;
+    bool own_arena = false;
+    float *w = nullptr, *D = nullptr, *r = nullptr, *m = nullptr;
+    int32_t* slot = nullptr;               // [K][slot_cap] row -> slot scratch map
+    int64_t slot_cap = 0;
+    bool own_slot = false;
+    cudaStream_t main = nullptr, side = nullptr, copy = nullptr;
+    bool own_streams = false;
+    std::vector<cudaEvent_t> ev_local, ev_merge;
+    std::vector<char> local_recorded, merge_unwaited;
+    bool D_valid = false;
+    int64_t merges = 0;
+    int form = HPSGD_FORM_REPLICA_CHANGE;  // what the workers carry: replica change or accumulated gradients
+    int fuse = 0;                          // carry a merge into the next batched local step
+    int pipeline = 0;                      // commit/reduce split on double-buffered replicas
+    float* wbuf[2] = {nullptr, nullptr};   // pipeline: global model of the current / other period
+    float* rbuf[2] = {nullptr, nullptr};   // pipeline: replica sets of the current / other period
+    int cur = 0;                           // pipeline: which buffers the current period trains on
+    std::vector<char> touched;             // pipeline: worker has made a local step this period
+    cudaEvent_t ev_commit = nullptr, ev_reduce = nullptr;
+    bool reduce_outstanding = false;
+    bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
+    int deferred_flags = 0;
+    std::vector<int> steps_in_period;      // local steps of each worker since the last merge request
+    bool deferred_all_single = false;      // every worker made exactly one step in the period the deferred merge closes
+    bool replicas_stale = false;           // replica rows not written by the implicit-replica kernel
+    int64_t launches = 0;
+    int sm_count = 148;
+    int sp_tensor = -1;                    // sparse-row tensor
+    int64_t sp_rows = 0, sp_cols = 0;
+    void* stage[2] = {nullptr, nullptr};   // staging of hpsgd_local_step_host
+    cudaEvent_t stage_copied[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
+    bool stage_used[2] = {false, false};
+    int stage_next = 0;
+    std::vector<EventPair> prof;           // profiling
+    double prof_ms[3] = {0, 0, 0};
+    int64_t prof_launches[3] = {0, 0, 0};
+} g;
+
+int check_async()
+{
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) return fail(HPSGD_E_CUDA, "CUDA error: %s", cudaGetErrorString(e));
+    return HPSGD_OK;
+}
+
+int64_t layout_of(const std::vector<int64_t>& sizes, std::vector<int64_t>* offsets, std::vector<int64_t>* starts)
+{
+    int64_t pos = 0, flat = 0;
+    for (int64_t s : sizes) {
+        if (offsets) offsets->push_back(pos);
+        if (starts) starts->push_back(flat);
+        pos += (s + kAlignElems - 1) / kAlignElems * kAlignElems;
+        flat += s;
+    }
+    return pos;
+}
+
+// Regions of the arena, in order: w | D | r[K] | m[K] | w2 | r2[K] | table | slot maps (the rest).
+struct ArenaPlan {
+    size_t w, D, r, m, w2, r2, table, slot, fixed;
+};
+
+ArenaPlan plan_arena(int64_t stride, int K, bool momentum, bool pipeline)
+{
+    ArenaPlan a{};
+    const size_t row = (size_t)stride * 4;
+    size_t pos = 0;
+    a.w = pos; pos += row;
+    a.D = pos; pos += row;
+    a.r = pos; pos += row * K;
+    a.m = pos; if (momentum) pos += row * K;
+    a.w2 = pos; if (pipeline) pos += row;
+    a.r2 = pos; if (pipeline) pos += row * K;
+    a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kAlignBytes);
+    a.slot = pos;
+    a.fixed = pos;
+    return a;
+}
+
+// Index range [o_lo, o_hi), in 8-element groups, of schedule chunk c.
+void chunk_range(int c, int64_t* o_lo, int64_t* o_hi)
+{
+    const int64_t n = g.P_pad / 8;
+    const int64_t grains = (n + kChunkGrain - 1) / kChunkGrain;
+    auto edge = [&](int k) { return std::min(n, grains * k / g.chunks * kChunkGrain); };
+    *o_lo = edge(c);
+    *o_hi = (c == g.chunks - 1) ? n : edge(c + 1);
+}
+
+// Grid of the hot kernels: one block per kHotThreads groups.
+int hot_grid(int64_t groups)
+{
+    return (int)std::min<int64_t>(kMaxGridX, std::max<int64_t>(1, (groups + kHotThreads - 1) / kHotThreads));
+}
+
+// Grid of the support kernels: enough blocks to cover `items`, capped at one full wave of
+// resident blocks (SM count x blocks the kernel can keep resident per SM).
+template <typename Kern>
+int grid_for(Kern kern, int64_t items, int64_t per_block)
+{
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0) != cudaSuccess || occ < 1) occ = 1;
+    const int64_t need = std::max<int64_t>(1, (items + per_block - 1) / per_block);
+    return (int)std::min<int64_t>(need, (int64_t)g.sm_count * occ);
+}
+
+// ---------------------------------------------------------------------------- profiling
+int prof_begin(cudaStream_t s, int kind, EventPair* ep)
+{
+    if (!g.profile) return HPSGD_OK;
+    ep->kind = kind;
+    CUDA_TRY(cudaEventCreate(&ep->a));
+    CUDA_TRY(cudaEventCreate(&ep->b));
+    CUDA_TRY(cudaEventRecord(ep->a, s));
+    return HPSGD_OK;
+}
+
+int prof_end(cudaStream_t s, EventPair* ep)
+{
+    if (!g.profile) return HPSGD_OK;
+    CUDA_TRY(cudaEventRecord(ep->b, s));
+    g.prof.push_back(*ep);
+    return HPSGD_OK;
+}
+
+int prof_resolve()
+{
+    for (EventPair& ep : g.prof) {
+        CUDA_TRY(cudaEventSynchronize(ep.b));
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, ep.a, ep.b));
+        g.prof_ms[ep.kind] += ms;
+        g.prof_launches[ep.kind] += 1;
+        cudaEventDestroy(ep.a);
+        cudaEventDestroy(ep.b);
+    }
+    g.prof.clear();
+    return HPSGD_OK;
+}
+
+int check_grad_ptr(const void* p, const char* what)
+{
+    if (!p) return fail(HPSGD_E_BADARG, "%s is NULL", what);
+    if (reinterpret_cast<uintptr_t>(p) % 32) return fail(HPSGD_E_BADARG, "%s is not 32-byte aligned", what);
+    return HPSGD_OK;
+}
+
+int check_desc(const hpsgd_grad_desc* d)
+{
+    if (!d) return fail(HPSGD_E_BADARG, "descriptor is NULL");
+    TRY(check_grad_ptr(d->dense, "dense gradient"));
+    if (d->n_rows < 0 || d->n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows %d out of range", d->n_rows);
+    if (d->n_rows > 0 && d->row_idx) TRY(check_grad_ptr(d->row_vals, "row_vals"));
+    return HPSGD_OK;
+}
+
+int need_init()
+{
+    if (!g.inited) return fail(HPSGD_E_STATE, "hpsgd_init has not been called");
+    return HPSGD_OK;
+}
+
+int check_worker(int worker)
+{
+    if (worker < 0 || worker >= g.K) return fail(HPSGD_E_BADARG, "worker %d outside [0, %d)", worker, g.K);
+    return HPSGD_OK;
+}
+
+int sync_all()
+{
+    CUDA_TRY(cudaStreamSynchronize(g.main));
+    CUDA_TRY(cudaStreamSynchronize(g.side));
+    if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
+    return HPSGD_OK;
+}
+
+int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; blocking
+{
+    const size_t row = (size_t)g.stride * 4;
+    CUDA_TRY(cudaMemsetAsync(g.D, 0, row, g.main));
+    if (g.m) CUDA_TRY(cudaMemsetAsync(g.m, 0, row * g.K, g.main));
+    if (g.pipeline) {
+        std::fill(g.touched.begin(), g.touched.end(), 0);      // replicas are w until their first step
+        g.reduce_outstanding = false;
+    } else {
+        const int64_t nvec = g.P_pad / 4;
+        clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
+        ++g.launches;
+        CUDA_TRY(cudaGetLastError());
+    }
+    CUDA_TRY(cudaStreamSynchronize(g.main));
+    g.D_valid = false;
+    g.merges = 0;
+    g.replicas_stale = false;
+    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 0);
+    std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
+    std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
+    return HPSGD_OK;
+}
+
+int make_chunk_events(int chunks)
+{
+    for (cudaEvent_t e : g.ev_local) cudaEventDestroy(e);
+    for (cudaEvent_t e : g.ev_merge) cudaEventDestroy(e);
+    g.ev_local.assign(chunks, nullptr);
+    g.ev_merge.assign(chunks, nullptr);
+    g.local_recorded.assign(chunks, 0);
+    g.merge_unwaited.assign(chunks, 0);
+    g.chunks = chunks;
+    for (int c = 0; c < chunks; ++c) {
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_local[c], cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_merge[c], cudaEventDisableTiming));
+    }
+    return HPSGD_OK;
+}
+
+GenParams gen_params(int worker, int step, int kind, double scale)
+{
+    GenParams gp{};
+    gp.key = g.key;
+    gp.step = (uint64_t)step;
+    gp.worker = (uint64_t)worker;
+    gp.kind = kind;
+    gp.scale_f = (float)scale;
+    gp.scale_d = scale;
+    if (g.sp_tensor >= 0) {
+        gp.sp_start = g.starts[g.sp_tensor];
+        gp.sp_rows = g.sp_rows;
+        gp.sp_cols = g.sp_cols;
+    }
+    return gp;
+}
+
+int check_gen_args(const void* out, int worker, int step, int kind)
+{
+    TRY(need_init());
+    TRY(check_grad_ptr(out, "output buffer"));
+    if (worker < 0 || worker >= 256) return fail(HPSGD_E_BADARG, "worker must be in [0, 256)");
+    if (step < 0 || step >= (1 << 20)) return fail(HPSGD_E_BADARG, "step must be in [0, 2^20)");
+    if (kind != HPSGD_GEN_UNIFORM && kind != HPSGD_GEN_GAUSS) return fail(HPSGD_E_BADARG, "unknown generator kind");
+    return HPSGD_OK;
+}
+
+void release_all()
+{
+    if (g.main) cudaStreamSynchronize(g.main);
+    if (g.side) cudaStreamSynchronize(g.side);
+    if (g.copy) cudaStreamSynchronize(g.copy);
+    for (EventPair& ep : g.prof) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+    for (cudaEvent_t e : g.ev_local) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : g.ev_merge) if (e) cudaEventDestroy(e);
+    if (g.ev_commit) cudaEventDestroy(g.ev_commit);
+    if (g.ev_reduce) cudaEventDestroy(g.ev_reduce);
+    for (int b = 0; b < 2; ++b) {
+        if (g.stage[b]) cudaFree(g.stage[b]);
+        if (g.stage_copied[b]) cudaEventDestroy(g.stage_copied[b]);
+        if (g.stage_free[b]) cudaEventDestroy(g.stage_free[b]);
+    }
+    if (g.copy) cudaStreamDestroy(g.copy);
+    if (g.own_streams) {
+        if (g.main) cudaStreamDestroy(g.main);
+        if (g.side) cudaStreamDestroy(g.side);
+    }
+    if (g.own_slot && g.slot) cudaFree(g.slot);
+    if (g.own_arena && g.arena) cudaFree(g.arena);
+    cudaGetLastError();
+    g = Ctx();
+}
+
+}  // namespace
