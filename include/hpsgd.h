@@ -191,7 +191,9 @@ size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows);
 /*
  * Lend device memory and streams for the next hpsgd_init.  `arena` (256-byte aligned,
  * `bytes` long) stays owned by the caller and must outlive hpsgd_destroy; pass NULL / 0
- * to let the library allocate.  main_stream / side_stream are cudaStream_t handles
+ * to let the library allocate.  No work of the caller (a fill, a copy) may still be pending
+ * on the arena when hpsgd_init runs: the library writes it on its own streams, which do not
+ * wait for the caller's.  main_stream / side_stream are cudaStream_t handles
  * owned by the caller (e.g. torch streams); pass NULL to let the library create its own.
  */
 int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream);

@@ -53,6 +53,7 @@ def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, pipelin
             nbytes = hp.hpsgd_arena_bytes(lay.P_pad, cfg.K, flags, rows)
             guard = 4096 if canary else 0
             buf = torch.full((nbytes + 2 * guard + 256,), 0xA5, dtype=torch.uint8, device=DEV)
+            torch.cuda.synchronize()     # the fill runs on torch's stream; the library works on its own
             base = buf.data_ptr() + guard
             base += (-base) % 256
             keep.update(buf=buf, base=base, nbytes=nbytes, guard=guard)

@@ -16,7 +16,7 @@ from tests import gpu_util as gu
 pytestmark = pytest.mark.gpu
 
 
-def run_full(cfg, T):
+def run_full(cfg, T, fuse):
     lay = cfg.layout
     K, P_pad = cfg.K, lay.P_pad
     bf16 = cfg.grad_dtype == "bf16"
@@ -28,11 +28,15 @@ def run_full(cfg, T):
     oracle = RefHPSGD(idx.size, K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
     oracle.set_global(cfg.initial_global(idx))
 
-    with gu.session(cfg, lend_arena=True, streams=True, canary=True):
+    with gu.session(cfg, fuse=fuse, lend_arena=True, streams=True, canary=True):
+        # one gradient buffer, refilled every round by the device generator: generator and consumers
+        # are all enqueued on the main stream, so no host synchronisation is needed (one would also
+        # launch a deferred merge on its own and keep the fused kernel from ever running)
         grads = torch.empty((K, P_pad), dtype=gdt, device=gu.DEV)
+        keep = []
+        hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)
         for t in range(T):
-            hp.hpsgd_synchronize()                   # the one gradient buffer is reused every round
-            descs, keep = [], []
+            descs = []
             for i in range(K):
                 hp.hpsgd_gen_grads(grads[i], i, t, kind, cfg.grad_scale)
                 if cfg.sparse:
@@ -50,6 +54,10 @@ def run_full(cfg, T):
                 oracle.local_step(i, cfg.stored_gradient(i, t, idx))
             oracle.sync_merge()
         hp.hpsgd_synchronize()
+        fused_launches = hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE_STEP)[1]
+        merge_launches = hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE)[1]
+        # the schedule under test really ran: T-1 merges inside fused kernels + the last one alone
+        assert (fused_launches, merge_launches) == ((T - 1, 1) if fuse else (0, T))
         got = {"w": gu.dev_gather(hp.hpsgd_get_global(), P_pad, pos),
                "D": gu.dev_gather(hp.hpsgd_get_pending(), P_pad, pos)}
         for i in (0, K // 2, K - 1):
@@ -64,10 +72,13 @@ def run_full(cfg, T):
     return idx, got, want
 
 
+@pytest.mark.parametrize("fuse", [1, 0, 2])
 @pytest.mark.parametrize("name", ["cfg4", "cfg5"])
-def test_full_size_sampled_parity(name):
+def test_full_size_sampled_parity(name, fuse):
+    """fuse = 1 is the configuration bench.py times by default; 0 (separate kernels on two
+    streams) and 2 (replicas left implicit) are its other schedules."""
     cfg = workloads.get(name)
-    idx, got, want = run_full(cfg, cfg.T)
+    idx, got, want = run_full(cfg, cfg.T, fuse)
     assert idx.size > 250_000
     for key in got:
         # parameters and replicas to 1e-6 relative (floor 1e-6); the momentum and pending-change
