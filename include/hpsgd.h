@@ -108,7 +108,8 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed);
  * device buffer of P_pad elements in the flat layout, fp32 or bf16 per
  * HPSGD_OPT_GRAD_DTYPE, 32-byte aligned, zero in the pads.  It is borrowed: keep it
  * valid and unchanged until the work has run (hpsgd_synchronize, or a stream wait on
- * the main stream).  Several local steps per worker between two merges are legal
+ * the main stream).  Its contents must be complete when the call is made, or be produced
+ * by work enqueued earlier on the main stream: the library does not wait for other streams.  Several local steps per worker between two merges are legal
  * (Section 3.2: several local trainings per synchronisation); a worker with none
  * contributes a zero change.  Enqueued on the main stream.
  */
@@ -191,9 +192,9 @@ size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows);
 /*
  * Lend device memory and streams for the next hpsgd_init.  `arena` (256-byte aligned,
  * `bytes` long) stays owned by the caller and must outlive hpsgd_destroy; pass NULL / 0
- * to let the library allocate.  No work of the caller (a fill, a copy) may still be pending
- * on the arena when hpsgd_init runs: the library writes it on its own streams, which do not
- * wait for the caller's.  main_stream / side_stream are cudaStream_t handles
+ * to let the library allocate.  hpsgd_init waits for all work on the device before it
+ * first writes a lent arena (the library works on its own streams, which do not otherwise wait
+ * for the caller's); after that the caller must leave the arena alone.  main_stream / side_stream are cudaStream_t handles
  * owned by the caller (e.g. torch streams); pass NULL to let the library create its own.
  */
 int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream);

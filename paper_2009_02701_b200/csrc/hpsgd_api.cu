@@ -102,6 +102,9 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     if (prop.major != 10)
         return fail(HPSGD_E_CUDA, "built for sm_100a only; device is sm_%d%d", prop.major, prop.minor);
 
+    // a lent arena may still be the target of the caller's own work on other streams
+    if (g_pending.arena) CUDA_TRY(cudaDeviceSynchronize());
+
     g = Ctx();
     g.sm_count = prop.multiProcessorCount;
     g.P = P; g.K = K; g.lr = lr; g.beta = momentum; g.seed = seed;
