@@ -190,22 +190,35 @@ def oracle_sample_run(cfg, seconds, sample_params=4_000_000, min_rounds=2, max_r
 
 
 def run_reference(args, cfg):
-    """--impl reference: the oracle, one bounded sample per step."""
-    for _ in range(max(0, args.warmup)):
-        oracle_sample_run(cfg, 0, sample_params=args.ref_sample, max_rounds=1)
-    t_total, units = 0.0, 0
-    desc = ""
-    for _ in range(args.steps):
-        eps, rounds, spent, desc, P = oracle_sample_run(cfg, 0, sample_params=args.ref_sample, max_rounds=1)
-        t_total += spent
-        units += cfg.K * P
-    value = units / t_total
+    """--impl reference: the CPU oracle as it stands; each step is one round (K local steps + one
+    merge) on a bounded sample of the workload, the first `--ref-sample` parameters."""
+    from oracle.ref import RefHPSGD
+    P = min(cfg.P, args.ref_sample)
+    idx = np.arange(P, dtype=np.int64)
+    o = RefHPSGD(P, cfg.K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+    o.set_global(cfg.initial_global(idx))
+    grads = [[cfg.stored_gradient(i, t, idx) for i in range(cfg.K)] for t in range(2)]   # untimed, as on the GPU
+
+    def one_round(t):
+        t0 = time.perf_counter()
+        for i in range(cfg.K):
+            o.local_step(i, grads[t % 2][i])
+        o.sync_merge()
+        return time.perf_counter() - t0
+
+    for t in range(max(0, args.warmup)):
+        one_round(t)
+    t_total = sum(one_round(args.warmup + t) for t in range(args.steps))
+    o.close()
+    value = cfg.K * P * args.steps / t_total
+    desc = ("first %d of %d parameters of %s, all K=%d workers, one round per step (local steps + merge; "
+            "sparse rows given as dense zeros), single thread" % (P, cfg.P, cfg.name, cfg.K))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic (counter-hash gradients)",
-        "config": workload_config(cfg, {"sample": "each step = one round on the first %d parameters" % min(cfg.P, args.ref_sample)}),
+        "config": workload_config(cfg, {"sample": "each step = one round on the first %d parameters" % P}),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
