@@ -1,0 +1,75 @@
+"""Random call sequences against the oracle: batched and per-worker local steps, merges
+(also back to back), synchronisations, option changes and checkpoints, under every schedule
+option.  Whatever the library defers, fuses or rebuilds internally, its state must equal the
+oracle's bit for bit."""
+import numpy as np
+import pytest
+
+import paper_2009_02701_b200 as hp
+from tests import gpu_util as gu
+from workloads.configs import Workload
+
+pytestmark = pytest.mark.gpu
+
+
+def compare(cfg, o, what):
+    w, D, rs, ms = gu.gpu_state(cfg)
+    gu.assert_bitwise(w, o.get_global(), "%s: global model" % what)
+    gu.assert_bitwise(D, o.get_pending(), "%s: pending change" % what)
+    for i in range(cfg.K):
+        gu.assert_bitwise(rs[i], o.get_replica(i), "%s: replica %d" % (what, i))
+        if cfg.momentum:
+            gu.assert_bitwise(ms[i], o.get_momentum(i), "%s: momentum %d" % (what, i))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_call_sequences(seed):
+    rng = np.random.default_rng(1000 + seed)
+    K = int(rng.choice([1, 2, 3, 4, 5, 8, 16]))
+    sizes = [int(x) for x in rng.integers(1, 20_000, size=int(rng.integers(1, 5)))]
+    momentum = float(rng.choice([0.0, 0.9]))
+    wd = float(rng.choice([0.0, 1e-3]))
+    pipeline = int(rng.random() < 0.25)
+    staleness = 1 if pipeline else int(rng.choice([0, 1]))
+    cfg = Workload("fuzz", K=K, sizes=tuple(sizes), T=0, lr=0.05, momentum=momentum, weight_decay=wd,
+                   seed=100 + seed, grad_kind="gauss", grad_scale=1e-2, staleness=staleness)
+    fuse = int(rng.choice([0, 1, 2]))
+    o = gu.oracle_for(cfg, staleness)
+    keep = []
+    step = 0
+    with gu.session(cfg, staleness=staleness, overlap=int(rng.choice([0, 1])), chunks=1 if pipeline else int(rng.choice([1, 3])),
+                    fuse=fuse, pipeline=pipeline, lend_arena=bool(rng.random() < 0.5), streams=bool(rng.random() < 0.5)):
+        for op_no in range(30):
+            op = rng.choice(["all", "all", "all", "some", "merge", "merge", "merge", "sync", "look", "chunks", "ckpt"])
+            if op == "all":
+                inputs = [gu.host_inputs(cfg, i, step) for i in range(K)]
+                stacked = np.stack([inp["padded"] for inp in inputs])
+                keep.append(gu.to_device(stacked.reshape(-1)))
+                hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
+                for i, inp in enumerate(inputs):
+                    o.local_step(i, inp["flat"])
+                step += 1
+            elif op == "some":
+                for i in rng.permutation(K)[:int(rng.integers(1, K + 1))]:
+                    inp = gu.host_inputs(cfg, int(i), step)
+                    gu.gpu_step(cfg, int(i), inp, keep)
+                    o.local_step(int(i), inp["flat"])
+                step += 1
+            elif op == "merge":
+                hp.hpsgd_sync_merge()
+                o.sync_merge()
+            elif op == "sync":
+                hp.hpsgd_synchronize()
+            elif op == "look":
+                compare(cfg, o, "seed %d after op %d" % (seed, op_no))
+            elif op == "chunks" and not pipeline:
+                hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, int(rng.choice([1, 2, 5])))
+                hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, int(rng.choice([0, 1, 2])))
+            elif op == "ckpt":
+                blob = np.empty(hp.hpsgd_state_bytes(), dtype=np.uint8)
+                hp.hpsgd_export_state(blob)
+                # wreck the live state, then restore it from the blob
+                hp.hpsgd_set_global_host(np.zeros(cfg.P, dtype=np.float32))
+                hp.hpsgd_import_state(blob)
+        compare(cfg, o, "seed %d at the end" % seed)
+    o.close()
