@@ -119,12 +119,13 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
     return check_async();
 }
 
-// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors: one memset over
-// the nw consecutive maps (every row: no slot, -1) and one scatter launch for all of them.
+// Build the row -> slot maps of workers [w0, w0 + nw) from their descriptors: one (strided)
+// memset over the nw maps (every row: no slot, -1) and one scatter launch for all of them.
 int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* gp)
 {
     int32_t* first = g.slot + (int64_t)w0 * g.slot_cap;
-    CUDA_TRY(cudaMemsetAsync(first, 0xFF, (size_t)g.slot_cap * 4 * nw, g.main));
+    // only the rows in use are reset: the maps are slot_cap entries apart, which can be far more
+    CUDA_TRY(cudaMemset2DAsync(first, (size_t)g.slot_cap * 4, 0xFF, (size_t)g.sp_rows * 4, nw, g.main));
     SlotBatch sb{};
     int32_t most = 0;
     for (int i = 0; i < nw; ++i) {
