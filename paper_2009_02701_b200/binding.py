@@ -217,13 +217,17 @@ def hpsgd_local_step_host(worker, host_grads):
     return _check(load().hpsgd_local_step_host(int(worker), _ptr(host_grads)))
 
 
+def _count(x):
+    """Number of elements of a numpy array or torch tensor."""
+    return int(x.numel()) if hasattr(x, "numel") else int(x.size)
+
+
 def hpsgd_set_global_host(host_w):
-    return _check(load().hpsgd_set_global_host(_ptr(host_w), int(host_w.size if hasattr(host_w, "size") and not callable(host_w.size) else host_w.numel())))
+    return _check(load().hpsgd_set_global_host(_ptr(host_w), _count(host_w)))
 
 
 def hpsgd_copy_global(host_out):
-    n = host_out.size if hasattr(host_out, "size") and not callable(host_out.size) else host_out.numel()
-    return _check(load().hpsgd_copy_global(_ptr(host_out), int(n)))
+    return _check(load().hpsgd_copy_global(_ptr(host_out), _count(host_out)))
 
 
 # ---- inspection ----------------------------------------------------------------------
