@@ -1,15 +1,18 @@
 """The allocation-free sparse-row step against the regular one.
 
-hpsgd_local_step_sparse_noalloc serves callers that cannot hand the library any device
-memory of their own choosing at call time (a process whose allocator already owns the
-whole GPU, or a latency-critical loop that must not hit cudaMalloc's device-wide
-synchronisation): its row -> slot scratch map is a fixed array inside the library.  The
-test runs the same two consecutive steps through it and through hpsgd_local_step_ex and
-requires bit-identical replicas and momenta; the second step uses a different set of
-active rows, so a map that kept the first call's entries would be caught.
+hpsgd_local_step_sparse_noalloc exists for programs that cannot allocate device memory at the
+moment they want to step: a server whose own allocator claimed the whole GPU at start-up, so
+that a cudaMalloc by anyone else simply fails; a latency-critical loop in which the device-wide
+synchronisation hidden in cudaMalloc / cudaFree would stall every other stream; a process held
+to a fixed memory budget.  For them the row -> slot scratch map of the sparse-row step is a
+fixed array inside the library image instead of a piece of an arena.
 
-This file is named to be collected last: if it fails under `pytest -x`, every other test
-has already run.
+The test runs the same two consecutive steps through that entry point and through
+hpsgd_local_step_ex and requires bit-identical replicas and momenta.  The second step uses a
+different set of active rows, so a map that still held the first call's entries would be caught.
+
+This file is named to be collected last: if it fails under `pytest -x`, every other test has
+already run.
 """
 import numpy as np
 import pytest
