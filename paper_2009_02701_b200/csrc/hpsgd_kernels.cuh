@@ -218,6 +218,49 @@ __global__ void scatter_slots_kernel(SlotBatch sb, int64_t rows)
 //   acc = (r_0 - w) + ... + (r_{K-1} - w) left to right ; Dnew = acc / K
 //   staleness 1: w += D (if a previous average exists) ; staleness 0: w += Dnew
 //   D = Dnew ; r_i = w
+// Left-to-right sum of replica changes for a run-time K: workers [i, i + N) are requested
+// together and then added in order.  start_changes also takes the first term, which opens the sum.
+template <int N>
+__device__ __forceinline__ void add_changes(f8& acc, const float* __restrict__ r, int64_t stride, int i,
+                                            int64_t e, const f8& wv)
+{
+    f8 rv[N];
+#pragma unroll
+    for (int b = 0; b < N; ++b) rv[b] = ld8(r + (int64_t)(i + b) * stride + e);
+#pragma unroll
+    for (int b = 0; b < N; ++b)
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
+}
+
+template <int N>
+__device__ __forceinline__ void start_changes(f8& acc, const float* __restrict__ r, int64_t stride, int64_t e,
+                                              const f8& wv)
+{
+    f8 rv[N];
+#pragma unroll
+    for (int b = 0; b < N; ++b) rv[b] = ld8(r + (int64_t)b * stride + e);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(rv[0].v[q], wv.v[q]);
+#pragma unroll
+    for (int b = 1; b < N; ++b)
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
+}
+
+// acc = (r_0 - w) + (r_1 - w) + ... + (r_{K-1} - w), eight replicas in flight at a time.
+__device__ __forceinline__ void sum_changes(f8& acc, const float* __restrict__ r, int64_t stride, int K,
+                                            int64_t e, const f8& wv)
+{
+    int i;
+    if (K >= 8) { start_changes<8>(acc, r, stride, e, wv); i = 8; }
+    else if (K >= 4) { start_changes<4>(acc, r, stride, e, wv); i = 4; }
+    else { start_changes<1>(acc, r, stride, e, wv); i = 1; }
+    for (; i + 8 <= K; i += 8) add_changes<8>(acc, r, stride, i, e, wv);
+    for (; i + 4 <= K; i += 4) add_changes<4>(acc, r, stride, i, e, wv);
+    for (; i < K; ++i) add_changes<1>(acc, r, stride, i, e, wv);
+}
+
 constexpr int kMergeApplyPending = 1;   // flags: a previous average exists (staleness 1)
 constexpr int kMergeImmediate = 2;      // flags: staleness 0
 
@@ -247,26 +290,7 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
 #pragma unroll
                 for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
         } else {
-            {
-                const f8 r0 = ld8(r + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
-            }
-            int i = 1;
-            for (; i + 4 <= K; i += 4) {
-                f8 rv[4];
-#pragma unroll
-                for (int b = 0; b < 4; ++b) rv[b] = ld8(r + (int64_t)(i + b) * stride + e);
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
-            }
-            for (; i < K; ++i) {
-                const f8 ri = ld8(r + (int64_t)i * stride + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
-            }
+            sum_changes(acc, r, stride, K, e, wv);
         }
         f8 dnew, wn;
 #pragma unroll
@@ -535,26 +559,7 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
 #pragma unroll
                 for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
         } else {
-            {
-                const f8 r0 = ld8(r + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
-            }
-            int i = 1;
-            for (; i + 4 <= K; i += 4) {
-                f8 rv[4];
-#pragma unroll
-                for (int b = 0; b < 4; ++b) rv[b] = ld8(r + (int64_t)(i + b) * stride + e);
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
-            }
-            for (; i < K; ++i) {
-                const f8 ri = ld8(r + (int64_t)i * stride + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
-            }
+            sum_changes(acc, r, stride, K, e, wv);
         }
         f8 dnew, wn;
 #pragma unroll
