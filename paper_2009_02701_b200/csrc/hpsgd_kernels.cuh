@@ -366,7 +366,17 @@ reduce_kernel(const float* __restrict__ w, float* __restrict__ D, ReducePtrs rp,
 #pragma unroll
                 for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
             }
-            for (int i = 1; i < K; ++i) {
+            int i = 1;
+            for (; i + 4 <= K; i += 4) {
+                f8 rv[4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) rv[b] = ld8(rp.src[i + b] + e);
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
+            }
+            for (; i < K; ++i) {
                 const f8 ri = ld8(rp.src[i] + e);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
