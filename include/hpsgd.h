@@ -131,7 +131,8 @@ int hpsgd_sync_merge(void);
 
 /*
  * Wait for all enqueued work and return the device pointer to w (P_pad floats, flat
- * layout, library-owned, valid until hpsgd_destroy).  The pending change D is NOT
+ * layout, library-owned, valid until hpsgd_destroy; with hpsgd_set_pipeline the global model
+ * alternates between two buffers, so ask again after every hpsgd_sync_merge).  The pending change D is NOT
  * flushed into it: after T merges w holds the changes of rounds 0..T-2 (one-
  * synchronisation delay).  Returns NULL on error.
  */
