@@ -109,9 +109,10 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed);
  * HPSGD_OPT_GRAD_DTYPE, 32-byte aligned, zero in the pads.  It is borrowed: keep it
  * valid and unchanged until the work has run (hpsgd_synchronize, or a stream wait on
  * the main stream).  Its contents must be complete when the call is made, or be produced
- * by work enqueued earlier on the main stream: the library does not wait for other streams.  Several local steps per worker between two merges are legal
- * (Section 3.2: several local trainings per synchronisation); a worker with none
- * contributes a zero change.  Enqueued on the main stream.
+ * by work enqueued earlier on the main stream: the library does not wait for other
+ * streams.  Several local steps per worker between two merges are legal (Section 3.2:
+ * several local trainings per synchronisation); a worker with none contributes a zero
+ * change.  Enqueued on the main stream.
  */
 int hpsgd_local_step(int worker, const void* grads);
 
