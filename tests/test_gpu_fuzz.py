@@ -73,3 +73,54 @@ def test_random_call_sequences(seed):
                 hp.hpsgd_import_state(blob)
         compare(cfg, o, "seed %d at the end" % seed)
     o.close()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_call_sequences_gradient_accumulation_form(seed):
+    """The same idea for Algorithms 2/3 as printed (explicit accumulated gradients)."""
+    from oracle.ref import RefHPSGDAccum
+    rng = np.random.default_rng(5000 + seed)
+    K = int(rng.choice([1, 3, 4, 8, 16]))
+    sizes = [int(x) for x in rng.integers(1, 20_000, size=int(rng.integers(1, 4)))]
+    cfg = Workload("fuzz_acc", K=K, sizes=tuple(sizes), T=0, lr=0.05, momentum=0.0, weight_decay=0.0,
+                   seed=200 + seed, grad_kind="uniform", grad_scale=1e-2)
+    o = RefHPSGDAccum(cfg.P, K, cfg.lr)
+    o.set_global(cfg.initial_global())
+    keep = []
+    step = 0
+
+    def look(what):
+        w, ghat, rs, accs = gu.gpu_state(cfg)
+        gu.assert_bitwise(w, o.get_global(), what + ": global model")
+        gu.assert_bitwise(ghat, o.get_synced(), what + ": AllReduce result")
+        for i in range(K):
+            gu.assert_bitwise(rs[i], o.get_replica(i), what + ": replica %d" % i)
+            gu.assert_bitwise(accs[i], o.get_accumulated(i), what + ": accumulated gradient %d" % i)
+
+    with gu.session(cfg, overlap=int(rng.choice([0, 1])), chunks=int(rng.choice([1, 3])), fuse=int(rng.choice([0, 1])),
+                    form=hp.HPSGD_FORM_GRADIENT_ACCUMULATION):
+        for op_no in range(25):
+            op = rng.choice(["all", "all", "some", "merge", "merge", "sync", "look"])
+            if op == "all":
+                inputs = [gu.host_inputs(cfg, i, step) for i in range(K)]
+                stacked = np.stack([inp["padded"] for inp in inputs])
+                keep.append(gu.to_device(stacked.reshape(-1)))
+                hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
+                for i, inp in enumerate(inputs):
+                    o.local_step(i, inp["flat"])
+                step += 1
+            elif op == "some":
+                for i in rng.permutation(K)[:int(rng.integers(1, K + 1))]:
+                    inp = gu.host_inputs(cfg, int(i), step)
+                    gu.gpu_step(cfg, int(i), inp, keep)
+                    o.local_step(int(i), inp["flat"])
+                step += 1
+            elif op == "merge":
+                hp.hpsgd_sync_merge()
+                o.sync_merge()
+            elif op == "sync":
+                hp.hpsgd_synchronize()
+            else:
+                look("seed %d after op %d" % (seed, op_no))
+        look("seed %d at the end" % seed)
+    o.close()
