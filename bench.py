@@ -285,8 +285,13 @@ def aggregate(dist, device, elapsed_ms, units):
 def run_gpu(args, cfg):
     import torch
     import paper_2009_02701_b200 as hp
+    from paper_2009_02701_b200 import build as cuda_build
 
     rank, world, local_rank, dist = dist_setup(args.gpus)
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        cuda_build.build()              # no-op when the in-tree library is up to date
+    if dist is not None:
+        dist.barrier()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     lay = cfg.layout

@@ -102,3 +102,15 @@ def test_product_code_never_touches_the_oracle():
         if f.endswith((".py", ".cpp")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2009_02701_b200" not in text and "libhpsgd.so" not in text
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 and as C++ with no other include."""
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "hpsgd.h"\n'
+                   'int probe(void) { hpsgd_grad_desc d = {0, 0, 0, 0}; (void)d; '
+                   'return (int)sizeof(hpsgd_status) + HPSGD_OPT_FUSE + HPSGD_NOALLOC_MAX_ROWS; }\n')
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)], check=True)
+    subprocess.run(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
