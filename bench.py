@@ -288,12 +288,12 @@ def run_gpu(args, cfg):
     from paper_2009_02701_b200 import build as cuda_build
 
     rank, world, local_rank, dist = dist_setup(args.gpus)
-    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if local_rank == 0:
         cuda_build.build()              # no-op when the in-tree library is up to date
     if dist is not None:
         dist.barrier()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
     lay = cfg.layout
     K, P, P_pad = cfg.K, cfg.P, lay.P_pad
     bf16 = cfg.grad_dtype == "bf16"
