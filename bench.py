@@ -288,8 +288,11 @@ def run_gpu(args, cfg):
     from paper_2009_02701_b200 import build as cuda_build
 
     rank, world, local_rank, dist = dist_setup(args.gpus)
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    # one GPU per rank; HPSGD_BENCH_DEVICE pins every rank to one device (single-GPU test runs of the
+    # multi-rank code path: the ranks are independent replicas and never wait for each other)
+    device_index = int(os.environ.get("HPSGD_BENCH_DEVICE", local_rank))
+    torch.cuda.set_device(device_index)
+    dev = torch.device("cuda", device_index)
     if local_rank == 0:
         cuda_build.build()              # no-op when the in-tree library is up to date
     if dist is not None:
@@ -367,7 +370,7 @@ def run_gpu(args, cfg):
         hp.hpsgd_sync_merge()
 
     # ---- warm-up, then the timed region (the clock sampler needs a moment to start)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(device_index)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
