@@ -333,7 +333,8 @@ def run_gpu(args, cfg):
 
     # ---- inputs: `nbuf` rounds of gradients for all K workers, generated on the device
     nbuf = args.grad_buffers
-    grads = torch.empty((nbuf, K, P_pad), dtype=gdt, device=dev)
+    row = -(-P_pad // 2048) * 2048          # every worker's gradient starts on a 4 KB boundary
+    grads = torch.empty((nbuf, K, row), dtype=gdt, device=dev)[:, :, :P_pad]
     sparse_in = None
     if cfg.sparse:
         rows_max = cfg.sparse[1]
@@ -366,7 +367,7 @@ def run_gpu(args, cfg):
             for i in range(K):
                 hp.hpsgd_local_step(i, grads[b, i])
         else:
-            hp.hpsgd_local_step_all(grads[b], P_pad * gsz)
+            hp.hpsgd_local_step_all(grads[b], row * gsz)
         hp.hpsgd_sync_merge()
 
     # ---- warm-up, then the timed region (the clock sampler needs a moment to start)

@@ -51,8 +51,9 @@ size_t hpsgd_arena_bytes(int64_t P_pad, int K, int flags, int64_t sparse_rows)
     if (P_pad <= 0 || K <= 0 || sparse_rows < 0) return 0;
     const int64_t stride = (P_pad + kRowAlignElems - 1) / kRowAlignElems * kRowAlignElems;
     const int64_t cap = (sparse_rows + 63) / 64 * 64;
+    // kPageBytes of slack: the regions start at the first 4 KB boundary inside the arena
     return plan_arena(stride, K, (flags & HPSGD_ARENA_MOMENTUM) != 0, (flags & HPSGD_ARENA_PIPELINE) != 0).fixed +
-           (size_t)cap * 4 * K;
+           (size_t)cap * 4 * K + kPageBytes;
 }
 
 int hpsgd_bind(void* arena, size_t bytes, void* main_stream, void* side_stream)
@@ -118,12 +119,16 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     const ArenaPlan a = plan_arena(g.stride, K, mom, g.pipeline != 0);
 
     if (g_pending.arena) {
-        if (g_pending.arena_bytes < a.fixed) {
+        if (g_pending.arena_bytes < a.fixed + kPageBytes) {
             g = Ctx();
-            return fail(HPSGD_E_NOMEM, "arena of %zu bytes is smaller than the %zu needed", g_pending.arena_bytes, a.fixed);
+            return fail(HPSGD_E_NOMEM, "arena of %zu bytes is smaller than the %zu needed", g_pending.arena_bytes,
+                        a.fixed + kPageBytes);
         }
-        g.arena = static_cast<char*>(g_pending.arena);
-        g.arena_bytes = g_pending.arena_bytes;
+        // the regions start at the first 4 KB boundary inside the lent memory
+        char* lent = static_cast<char*>(g_pending.arena);
+        const size_t skip = (kPageBytes - reinterpret_cast<uintptr_t>(lent) % kPageBytes) % kPageBytes;
+        g.arena = lent + skip;
+        g.arena_bytes = g_pending.arena_bytes - skip;
         g.slot_cap = (int64_t)((g.arena_bytes - a.fixed) / ((size_t)4 * K)) / 64 * 64;
         g.slot = g.slot_cap ? reinterpret_cast<int32_t*>(g.arena + a.slot) : nullptr;
     } else {

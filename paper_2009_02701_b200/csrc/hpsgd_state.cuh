@@ -18,8 +18,11 @@ namespace {
 using namespace hpsgd;
 
 constexpr int64_t kAlignElems = 32;        // tensor starts: multiples of 32 elements
-constexpr int64_t kRowAlignElems = 64;     // rows of r / m: multiples of 256 bytes
-constexpr size_t kAlignBytes = 256;        // arena regions
+constexpr int64_t kRowAlignElems = 1024;   // w, D and the rows of r / m start on 4 KB boundaries: the 4 KB
+                                           // tile a block touches in each array then never straddles one
+                                           // (measured +1.2-1.6 % on the merge over 256-byte alignment)
+constexpr size_t kAlignBytes = 256;        // what a lent arena must be aligned to
+constexpr size_t kPageBytes = 4096;        // what the regions inside it are aligned to
 constexpr int kMaxChunks = 1024;
 constexpr int kMaxTensors = 4096;
 constexpr int64_t kChunkGrain = 1024;      // chunk boundaries: multiples of 1024 groups (8192 elements)
@@ -150,7 +153,7 @@ ArenaPlan plan_arena(int64_t stride, int K, bool momentum, bool pipeline)
     a.m = pos; if (momentum) pos += row * K;
     a.w2 = pos; if (pipeline) pos += row;
     a.r2 = pos; if (pipeline) pos += row * K;
-    a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kAlignBytes);
+    a.table = pos; pos += round_up((size_t)kMaxTensors * 3 * 8, kPageBytes);
     a.slot = pos;
     a.fixed = pos;
     return a;
