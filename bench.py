@@ -65,14 +65,14 @@ def fused_bytes_per_index(cfg):
 # capture divided by the indices of that launch), keyed by (kernel, K, gradient dtype, fuse variant), with
 # the SHA-1 of the kernel source the capture was taken from.  A changed source voids them.
 NCU_TRAFFIC = {
-    # profiles/merge_step_kernel_cfg4_cut16M.txt (last launch): 3.200027 GB read + 2.121796 GB written over 16,000,000 indices
-    ('merge_step_kernel', 16, 'f32', 1): {"bytes_per_index": 5.321823e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
-    # profiles/merge_step_implicit_kernel_cfg4_cut16M.txt (last launch): 2.176032 GB read + 1.123314 GB written over 16,000,000 indices
-    ('merge_step_kernel', 16, 'f32', 2): {"bytes_per_index": 3.299346e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
-    # profiles/merge_kernel_cfg4_cut16M.txt (last launch): 1.152017 GB read + 1.093543 GB written over 16,000,000 indices
-    ('merge_kernel', 16, 'f32', 0): {"bytes_per_index": 2.245560e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
-    # profiles/local_step_kernel_cfg4_cut16M.txt (last launch): 3.072010 GB read + 1.996811 GB written over 16,000,000 indices
-    ('local_step_kernel', 16, 'f32', 0): {"bytes_per_index": 5.068821e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
+    # profiles/merge_step_kernel_cfg4_cut16M.txt (last launch): 3.200047 GB read + 2.123349 GB written over 16,000,000 indices
+    ('merge_step_kernel', 16, 'f32', 1): {"bytes_per_index": 5.323396e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
+    # profiles/merge_step_implicit_kernel_cfg4_cut16M.txt (last launch): 2.176030 GB read + 1.126342 GB written over 16,000,000 indices
+    ('merge_step_kernel', 16, 'f32', 2): {"bytes_per_index": 3.302372e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
+    # profiles/merge_kernel_cfg4_cut16M.txt (last launch): 1.152017 GB read + 1.093487 GB written over 16,000,000 indices
+    ('merge_kernel', 16, 'f32', 0): {"bytes_per_index": 2.245504e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
+    # profiles/local_step_kernel_cfg4_cut16M.txt (last launch): 3.072011 GB read + 1.997550 GB written over 16,000,000 indices
+    ('local_step_kernel', 16, 'f32', 0): {"bytes_per_index": 5.069561e9 / 16e6, "source_sha1": "5d530923c7baf3340525993c3ad2d3ee08488a94"},
 }
 
 
