@@ -518,14 +518,18 @@ def run_e2e(args, cfg, hp, torch, dev, grads, dist):
     host = [torch.empty(P_pad, dtype=grads.dtype).pin_memory() for _ in range(nhost)]
     for j in range(nhost):
         host[j].copy_(grads[0, j])
-    out = torch.empty(P, dtype=torch.float32).pin_memory()
+    out = [torch.empty(P, dtype=torch.float32).pin_memory() for _ in range(2)]
     torch.cuda.synchronize(dev)
+    counter = [0]
 
     def one_step():
+        # the read-back of step t runs beside the gradient uploads of step t+1 (PCIe is full duplex);
+        # two result buffers, so that a result stays readable while the next one is written
         for i in range(K):
             hp.hpsgd_local_step_host(i, host[i % nhost])
         hp.hpsgd_sync_merge()
-        hp.hpsgd_copy_global(out)
+        hp.hpsgd_copy_global_async(out[counter[0] % 2])
+        counter[0] += 1
 
     for _ in range(args.e2e_warmup):
         one_step()
@@ -538,10 +542,11 @@ def run_e2e(args, cfg, hp, torch, dev, grads, dist):
     t0 = time.perf_counter()
     for _ in range(args.e2e_steps):
         one_step()
+    hp.hpsgd_synchronize()                 # the last read-back is part of the timed region
     end.record()
     torch.cuda.synchronize(dev)
     wall_ms = (time.perf_counter() - t0) * 1e3
-    ms = max(start.elapsed_time(end), wall_ms)     # the device-to-host copy blocks the host
+    ms = max(start.elapsed_time(end), wall_ms)     # events on torch's stream do not see the library's streams
     job_ms, job_units = aggregate(dist, dev, ms, K * P * args.e2e_steps)
     if cfg.sparse:
         hp.hpsgd_set_sparse_segment(*cfg.sparse)

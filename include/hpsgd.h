@@ -309,6 +309,12 @@ int hpsgd_set_global_host(const float* host_w, int64_t n);
  * HOST array of n = P floats.  Blocking. */
 int hpsgd_copy_global(float* host_out, int64_t n);
 
+/* The same copy, enqueued behind the merges issued so far instead of waited for: it runs on a
+ * stream of its own, overlaps later local steps (and their host-to-device copies), and the next
+ * merge waits for it before it overwrites w.  host_out (pinned memory, else the call blocks) is
+ * complete after hpsgd_synchronize. */
+int hpsgd_copy_global_async(float* host_out, int64_t n);
+
 /* Device pointers (P_pad floats each) to worker's replica and momentum buffer (*m = NULL
  * when momentum == 0), and to the pending change D.  Any out pointer may be NULL.
  * Does not synchronise. */

@@ -61,6 +61,7 @@ SIGNATURES = {
     "hpsgd_local_step_host": (_ci, [_ci, _vp]),
     "hpsgd_set_global_host": (_ci, [_vp, _i64]),
     "hpsgd_copy_global": (_ci, [_vp, _i64]),
+    "hpsgd_copy_global_async": (_ci, [_vp, _i64]),
     "hpsgd_get_replica": (_ci, [_ci, _P(_vp), _P(_vp)]),
     "hpsgd_get_pending": (_ci, [_P(_vp)]),
     "hpsgd_state_bytes": (_sz, []),
@@ -228,6 +229,10 @@ def hpsgd_set_global_host(host_w):
 
 def hpsgd_copy_global(host_out):
     return _check(load().hpsgd_copy_global(_ptr(host_out), _count(host_out)))
+
+
+def hpsgd_copy_global_async(host_out):
+    return _check(load().hpsgd_copy_global_async(_ptr(host_out), _count(host_out)))
 
 
 # ---- inspection ----------------------------------------------------------------------

@@ -465,6 +465,29 @@ int hpsgd_copy_global(float* host_out, int64_t n)
     return HPSGD_OK;
 }
 
+int hpsgd_copy_global_async(float* host_out, int64_t n)
+{
+    TRY(need_init());
+    if (!host_out || n != g.P) return fail(HPSGD_E_BADARG, "need a host array of exactly P = %lld floats", (long long)g.P);
+    TRY(flush_deferred());
+    if (!g.d2h) {
+        CUDA_TRY(cudaStreamCreateWithFlags(&g.d2h, cudaStreamNonBlocking));
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_w_ready, cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&g.ev_d2h_done, cudaEventDisableTiming));
+    }
+    // w is last written by a merge: on the side stream, or on the main stream without overlap and
+    // in the pipelined schedule (its commit)
+    cudaStream_t writer = (g.overlap && !g.pipeline) ? g.side : g.main;
+    CUDA_TRY(cudaEventRecord(g.ev_w_ready, writer));
+    CUDA_TRY(cudaStreamWaitEvent(g.d2h, g.ev_w_ready, 0));
+    for (size_t t = 0; t < g.sizes.size(); ++t)
+        CUDA_TRY(cudaMemcpyAsync(host_out + g.starts[t], g.w + g.offsets[t], (size_t)g.sizes[t] * 4,
+                                 cudaMemcpyDeviceToHost, g.d2h));
+    CUDA_TRY(cudaEventRecord(g.ev_d2h_done, g.d2h));
+    g.d2h_outstanding = true;
+    return HPSGD_OK;
+}
+
 int hpsgd_get_replica(int worker, const float** r, const float** m)
 {
     TRY(need_init());

@@ -7,6 +7,13 @@
 
 namespace {
 
+// A host copy of w started by hpsgd_copy_global_async must finish before the stream `s` overwrites w.
+int wait_pending_d2h(cudaStream_t s)
+{
+    if (g.d2h_outstanding) CUDA_TRY(cudaStreamWaitEvent(s, g.ev_d2h_done, 0));
+    return HPSGD_OK;
+}
+
 // Rebuild replica rows that the implicit-replica kernel left stale: r_i = fma(-mu, m_i, w).
 int ensure_replicas()
 {
@@ -162,6 +169,7 @@ int enqueue_merge(int flags)
 {
     TRY(ensure_replicas());
     cudaStream_t s = g.overlap ? g.side : g.main;
+    TRY(wait_pending_d2h(s));
     for (int c = 0; c < g.chunks; ++c) {
         int64_t lo, hi;
         chunk_range(c, &lo, &hi);
@@ -210,6 +218,7 @@ int enqueue_pipelined_merge(int flags)
 {
     const int64_t n = g.P_pad / 8;
     const int nxt = g.cur ^ 1;
+    TRY(wait_pending_d2h(g.main));
     if (g.reduce_outstanding) {
         // the previous reduce still reads the buffers about to be written and produces the D read here
         CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_reduce, 0));
@@ -321,6 +330,7 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
 {
     const bool implicit = implicit_ok();
     if (!implicit) TRY(ensure_replicas());
+    TRY(wait_pending_d2h(g.main));
     for (int i = 0; i < g.K; ++i) g.steps_in_period[i] += 1;
     FusedLaunch L{};
     L.gp = gp;

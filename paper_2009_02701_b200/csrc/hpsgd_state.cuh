@@ -85,7 +85,9 @@ struct Ctx {
     int32_t* slot = nullptr;               // [K][slot_cap] row -> slot scratch map
     int64_t slot_cap = 0;
     bool own_slot = false;
-    cudaStream_t main = nullptr, side = nullptr, copy = nullptr;
+    cudaStream_t main = nullptr, side = nullptr, copy = nullptr, d2h = nullptr;
+    cudaEvent_t ev_w_ready = nullptr, ev_d2h_done = nullptr;   // hpsgd_copy_global_async
+    bool d2h_outstanding = false;
     bool own_streams = false;
     std::vector<cudaEvent_t> ev_local, ev_merge;
     std::vector<char> local_recorded, merge_unwaited;
@@ -253,6 +255,8 @@ int sync_all()
     CUDA_TRY(cudaStreamSynchronize(g.main));
     CUDA_TRY(cudaStreamSynchronize(g.side));
     if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
+    if (g.d2h) CUDA_TRY(cudaStreamSynchronize(g.d2h));
+    g.d2h_outstanding = false;
     return HPSGD_OK;
 }
 
@@ -328,6 +332,9 @@ void release_all()
     if (g.main) cudaStreamSynchronize(g.main);
     if (g.side) cudaStreamSynchronize(g.side);
     if (g.copy) cudaStreamSynchronize(g.copy);
+    if (g.d2h) { cudaStreamSynchronize(g.d2h); cudaStreamDestroy(g.d2h); }
+    if (g.ev_w_ready) cudaEventDestroy(g.ev_w_ready);
+    if (g.ev_d2h_done) cudaEventDestroy(g.ev_d2h_done);
     for (EventPair& ep : g.prof) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
     for (cudaEvent_t e : g.ev_local) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : g.ev_merge) if (e) cudaEventDestroy(e);

@@ -478,3 +478,30 @@ def test_implicit_replicas_are_rebuilt_on_demand():
         for i in range(cfg.K):
             gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d" % i)
             gu.assert_bitwise(ms[i], o.get_momentum(i), "momentum %d" % i)
+
+
+@pytest.mark.parametrize("mode", ["two_streams", "one_stream", "fuse", "pipeline"])
+def test_async_host_copy_sees_the_model_of_its_merge(mode):
+    """hpsgd_copy_global_async after merge t must deliver w as of merge t, although later local
+    steps and merges are enqueued before anything is waited for."""
+    cfg = small("d2h", 4, [60_000, 99], T=5, momentum=0.9)
+    kw = dict(overlap=0 if mode == "one_stream" else 1, fuse=int(mode == "fuse"), pipeline=int(mode == "pipeline"))
+    o = gu.oracle_for(cfg)
+    outs = [torch.empty(cfg.P, dtype=torch.float32).pin_memory() for _ in range(cfg.T)]
+    want = []
+    with gu.session(cfg, **kw):
+        keep = []
+        for t in range(cfg.T):
+            inputs = [gu.host_inputs(cfg, i, t) for i in range(cfg.K)]
+            stacked = np.stack([inp["padded"] for inp in inputs])
+            keep.append(gu.to_device(stacked.reshape(-1)))
+            hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
+            for i, inp in enumerate(inputs):
+                o.local_step(i, inp["flat"])
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+            hp.hpsgd_copy_global_async(outs[t])
+            want.append(o.get_global())
+        hp.hpsgd_synchronize()
+        for t in range(cfg.T):
+            gu.assert_bitwise(outs[t].numpy(), want[t], "host copy taken after merge %d" % t)
