@@ -58,6 +58,15 @@ def run_full(cfg, T, fuse):
         merge_launches = hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE)[1]
         # the schedule under test really ran: T-1 merges inside fused kernels + the last one alone
         assert (fused_launches, merge_launches) == ((T - 1, 1) if fuse else (0, T))
+        # properties that hold at every one of the K x P elements, checked on the device: the run
+        # ends with a merge, so every replica is a clone of w, and nothing is NaN or infinite
+        w_all = torch.as_tensor(gu._RawDeviceArray(hp.hpsgd_get_global(), P_pad, "<f4"), device=gu.DEV)
+        assert bool(torch.isfinite(w_all).all())
+        for i in range(K):
+            r_i, m_i = hp.hpsgd_get_replica(i)
+            assert torch.equal(torch.as_tensor(gu._RawDeviceArray(r_i, P_pad, "<f4"), device=gu.DEV), w_all), \
+                "replica %d is not a clone of the global model after the last merge" % i
+            assert bool(torch.isfinite(torch.as_tensor(gu._RawDeviceArray(m_i, P_pad, "<f4"), device=gu.DEV)).all())
         got = {"w": gu.dev_gather(hp.hpsgd_get_global(), P_pad, pos),
                "D": gu.dev_gather(hp.hpsgd_get_pending(), P_pad, pos)}
         for i in (0, K // 2, K - 1):
