@@ -16,7 +16,7 @@ from tests import gpu_util as gu
 pytestmark = pytest.mark.gpu
 
 
-def run_full(cfg, T, fuse):
+def run_full(cfg, T, fuse, pipeline=0):
     lay = cfg.layout
     K, P_pad = cfg.K, lay.P_pad
     bf16 = cfg.grad_dtype == "bf16"
@@ -28,7 +28,7 @@ def run_full(cfg, T, fuse):
     oracle = RefHPSGD(idx.size, K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
     oracle.set_global(cfg.initial_global(idx))
 
-    with gu.session(cfg, fuse=fuse, lend_arena=True, streams=True, canary=True):
+    with gu.session(cfg, fuse=fuse, pipeline=pipeline, lend_arena=True, streams=True, canary=True):
         # one gradient buffer, refilled every round by the device generator: generator and consumers
         # are all enqueued on the main stream, so no host synchronisation is needed (one would also
         # launch a deferred merge on its own and keep the fused kernel from ever running)
@@ -57,7 +57,10 @@ def run_full(cfg, T, fuse):
         fused_launches = hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE_STEP)[1]
         merge_launches = hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE)[1]
         # the schedule under test really ran: T-1 merges inside fused kernels + the last one alone
-        assert (fused_launches, merge_launches) == ((T - 1, 1) if fuse else (0, T))
+        if pipeline:
+            assert (fused_launches, merge_launches) == (0, 2 * T)       # one commit and one reduce per merge
+        else:
+            assert (fused_launches, merge_launches) == ((T - 1, 1) if fuse else (0, T))
         # properties that hold at every one of the K x P elements, checked on the device: the run
         # ends with a merge, so every replica is a clone of w, and nothing is NaN or infinite
         w_all = torch.as_tensor(gu._RawDeviceArray(hp.hpsgd_get_global(), P_pad, "<f4"), device=gu.DEV)
@@ -98,3 +101,12 @@ def test_full_size_sampled_parity(name, fuse):
         equal = np.mean(got[key].view(np.uint32) == want[key].view(np.uint32))
         # device and host log/cos may round a Gaussian differently once in ~1e8 draws
         assert equal >= 0.999, "%s: only %.6f of the sample is bit-equal" % (key, equal)
+
+
+def test_full_size_sampled_parity_pipelined_schedule():
+    """cfg4 under the paper's timeline: commit on the main stream, reduce on the side stream."""
+    cfg = workloads.get("cfg4")
+    idx, got, want = run_full(cfg, cfg.T, 0, pipeline=1)
+    for key in got:
+        assert np.array_equal(got[key].view(np.uint32), want[key].view(np.uint32)) or \
+            gu.max_rel_err(got[key], want[key], floor=1e-6 if key[0] in "wr" else 1e-9) <= 1e-6, key
