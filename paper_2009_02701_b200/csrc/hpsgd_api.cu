@@ -475,10 +475,11 @@ int hpsgd_copy_global_async(float* host_out, int64_t n)
         CUDA_TRY(cudaEventCreateWithFlags(&g.ev_w_ready, cudaEventDisableTiming));
         CUDA_TRY(cudaEventCreateWithFlags(&g.ev_d2h_done, cudaEventDisableTiming));
     }
-    // w is last written by a merge: on the side stream, or on the main stream without overlap and
-    // in the pipelined schedule (its commit)
-    cudaStream_t writer = (g.overlap && !g.pipeline) ? g.side : g.main;
-    CUDA_TRY(cudaEventRecord(g.ev_w_ready, writer));
+    // w is last written by a merge on the side stream, or on the main stream (no overlap, a fused
+    // merge + step kernel, the commit of the pipelined schedule): the copy waits for both
+    CUDA_TRY(cudaEventRecord(g.ev_w_ready, g.main));
+    CUDA_TRY(cudaStreamWaitEvent(g.d2h, g.ev_w_ready, 0));
+    CUDA_TRY(cudaEventRecord(g.ev_w_ready, g.side));
     CUDA_TRY(cudaStreamWaitEvent(g.d2h, g.ev_w_ready, 0));
     for (size_t t = 0; t < g.sizes.size(); ++t)
         CUDA_TRY(cudaMemcpyAsync(host_out + g.starts[t], g.w + g.offsets[t], (size_t)g.sizes[t] * 4,

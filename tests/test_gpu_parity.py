@@ -505,3 +505,28 @@ def test_async_host_copy_sees_the_model_of_its_merge(mode):
         hp.hpsgd_synchronize()
         for t in range(cfg.T):
             gu.assert_bitwise(outs[t].numpy(), want[t], "host copy taken after merge %d" % t)
+
+
+def test_async_host_copy_after_a_fused_kernel():
+    """The fused merge + step kernel writes w on the main stream; a host copy requested right
+    after it (before the next merge) must wait for it."""
+    cfg = small("d2h_fused", 8, [400_000], T=4, momentum=0.9)
+    o = gu.oracle_for(cfg)
+    outs = [torch.empty(cfg.P, dtype=torch.float32).pin_memory() for _ in range(cfg.T)]
+    want = []
+    with gu.session(cfg, fuse=1):
+        keep = []
+        for t in range(cfg.T):
+            inputs = [gu.host_inputs(cfg, i, t) for i in range(cfg.K)]
+            stacked = np.stack([inp["padded"] for inp in inputs])
+            keep.append(gu.to_device(stacked.reshape(-1)))
+            hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)     # carries merge t-1 from round 1 on
+            for i, inp in enumerate(inputs):
+                o.local_step(i, inp["flat"])
+            hp.hpsgd_copy_global_async(outs[t])                          # w as of merge t-1
+            want.append(o.get_global())
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+        hp.hpsgd_synchronize()
+        for t in range(cfg.T):
+            gu.assert_bitwise(outs[t].numpy(), want[t], "host copy taken after the step of round %d" % t)
