@@ -199,11 +199,14 @@ int prof_begin(cudaStream_t s, int kind, EventPair* ep)
     return HPSGD_OK;
 }
 
+int prof_resolve();
+
 int prof_end(cudaStream_t s, EventPair* ep)
 {
     if (!g.profile) return HPSGD_OK;
     CUDA_TRY(cudaEventRecord(ep->b, s));
     g.prof.push_back(*ep);
+    if (g.prof.size() >= 8192) return prof_resolve();   // bound the number of live events (waits for them)
     return HPSGD_OK;
 }
 
