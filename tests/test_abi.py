@@ -114,3 +114,25 @@ def test_header_is_plain_c(tmp_path):
     inc = os.path.join(ROOT, "include")
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)], check=True)
     subprocess.run(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
+
+
+def test_layout_matches_the_workload_helper_on_random_size_lists():
+    """Two independent implementations of the flat layout (the library's and the input module's)."""
+    import numpy as np
+    from workloads.configs import Layout
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        sizes = [int(x) for x in rng.integers(1, 5000, size=int(rng.integers(1, 40)))]
+        pad, off = hp.hpsgd_layout_padded(sizes)
+        lay = Layout(sizes)
+        assert (pad, off) == (lay.P_pad, lay.offsets)
+        assert all(o % 32 == 0 for o in off) and pad % 32 == 0
+        assert all(off[i + 1] - off[i] >= sizes[i] for i in range(len(sizes) - 1))
+        # the arena holds at least w, D and K rows of P_pad floats (+ K more with momentum or the
+        # pipelined schedule), whatever the padding
+        K = int(rng.integers(1, 20))
+        base = hp.hpsgd_arena_bytes(pad, K, 0, 0)
+        assert base >= (K + 2) * pad * 4
+        assert hp.hpsgd_arena_bytes(pad, K, hp.HPSGD_ARENA_MOMENTUM, 0) - base >= K * pad * 4
+        assert hp.hpsgd_arena_bytes(pad, K, hp.HPSGD_ARENA_PIPELINE, 0) - base >= (K + 1) * pad * 4
+        assert hp.hpsgd_arena_bytes(pad, K, 0, 1000) - base >= 1000 * 4 * K
