@@ -317,7 +317,8 @@ int hpsgd_copy_global_async(float* host_out, int64_t n);
 
 /* Device pointers (P_pad floats each) to worker's replica and momentum buffer (*m = NULL
  * when momentum == 0), and to the pending change D.  Any out pointer may be NULL.
- * Does not synchronise. */
+ * Does not synchronise: call hpsgd_synchronize first, which also launches a deferred merge
+ * and rebuilds replica rows that HPSGD_OPT_FUSE = 2 left implicit. */
 int hpsgd_get_replica(int worker, const float** r, const float** m);
 int hpsgd_get_pending(const float** D);
 
