@@ -379,7 +379,7 @@ def run_gpu(args, cfg):
         one_round(t)
     hp.hpsgd_synchronize()
     hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)     # also launches a merge deferred by the warm-up
-    for kind in range(3):
+    for kind in range(4):
         hp.hpsgd_profile_read(kind)
     if dist is not None:
         dist.barrier()
@@ -401,7 +401,7 @@ def run_gpu(args, cfg):
     elapsed_ms = start.elapsed_time(end)
     launches = hp.hpsgd_launch_count() - launches0
     prof = {name: hp.hpsgd_profile_read(kind) for kind, name in
-            enumerate(("local_step_kernel", "merge_kernel", "merge_step_kernel"))}
+            enumerate(("local_step_kernel", "merge_kernel", "merge_step_kernel", "round_kernel"))}
     hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 0)
     units = K * P * args.steps
     job_ms, job_units = aggregate(dist, dev, elapsed_ms, units)
@@ -421,9 +421,10 @@ def run_gpu(args, cfg):
     per_round = {"local_step_kernel": grad_bytes + state_bytes,
                  # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
                  "merge_kernel": (12 + (K + 2) * 4) * P if args.pipeline else merge_bytes_per_index(cfg) * P,
-                 # fuse 2 with momentum: the replica rows are neither read nor written
-                 "merge_step_kernel": 16 * P + grad_bytes + (K * P * 8 if (args.fuse == 2 and cfg.momentum and K in (4, 8, 16))
-                                                             else state_bytes)}
+                 "merge_step_kernel": 16 * P + grad_bytes + state_bytes,
+                 # whole round in one kernel, one step per worker and period: no replica row is read
+                 # or written; w, D, K m, K g in and w, D, K m out
+                 "round_kernel": 16 * P + grad_bytes + (K * P * 8 if cfg.momentum else 0)}
     kernels = {}
     for name, (ms, n) in prof.items():
         if n == 0:
@@ -440,8 +441,9 @@ def run_gpu(args, cfg):
                 "traffic": ncu_traffic(dominant, cfg, args.fuse) if (args.chunks == 1 and not args.per_worker) else None,
                 "peak_source": peak_src, "nominal_peak": NOMINAL_HBM_GBS, "kernels": kernels,
                 "note": "CUDA event pairs around each launch on its own stream inside the timed region; "
-                        "a fused merge_step_kernel launch moves 16 + K*(local step bytes) per index, "
-                        "8K fewer than the merge and local-step launches it replaces"}
+                        "bytes are the ones the launch actually moves: round_kernel (local steps + merge in one "
+                        "pass, replicas never stored) 16 + K*(g + 8) per index with momentum, merge_step_kernel "
+                        "16 + K*(g + 16), merge_kernel (2K + 4)*4, local_step_kernel K*(g + 16)"}
     moved = sum(k["algorithmic_bytes_per_launch"] * k["launches"] for k in kernels.values())
     roofline["round_achieved"] = moved / (elapsed_ms * 1e-3) / 1e9
     roofline["round_frac"] = roofline["round_achieved"] / peak
@@ -454,7 +456,7 @@ def run_gpu(args, cfg):
         for name, pipe, fuse in (("separate merge and local-step kernels on two streams", 0, 0),
                                  ("pipelined commit + reduce on double-buffered replicas", 1, 0),
                                  ("merge fused into the next local step", 0, 1),
-                                 ("fused, replicas implicit (recomputed from momentum)", 0, 2)):
+                                 ("one kernel per round (local steps + merge), replicas never stored", 0, 2)):
             if (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
                 continue
             setup(pipe, fuse, 1)
@@ -564,9 +566,10 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=workloads.names())
     ap.add_argument("--overlap", type=int, default=1)
     ap.add_argument("--chunks", type=int, default=1)
-    ap.add_argument("--fuse", type=int, default=1,
-                    help="1: carry each merge into the next batched local step (one kernel); "
-                         "2: also leave the replicas implicit where fma(-mu, m, w) reproduces them; 0: separate kernels")
+    ap.add_argument("--fuse", type=int, default=2,
+                    help="2: one kernel per round (the batched local step runs inside the kernel of the merge that "
+                         "follows it, replicas never stored); 1: carry each merge into the next batched local step; "
+                         "0: separate kernels on two streams")
     ap.add_argument("--pipeline", type=int, default=0,
                     help="paper timeline: commit on the main stream, K-way reduce on the side stream, double-buffered replicas")
     ap.add_argument("--other-schedule-steps", type=int, default=20,

@@ -41,7 +41,7 @@ typedef enum hpsgd_status {
     HPSGD_E_STATE = -2,       /* call not legal in the current state (e.g. before hpsgd_init) */
     HPSGD_E_NOMEM = -3,       /* arena too small or device allocation failed */
     HPSGD_E_CUDA = -4,        /* a CUDA call failed; see hpsgd_last_error() */
-    HPSGD_E_TIMEOUT = -5,     /* a bounded device-side wait gave up */
+    HPSGD_E_TIMEOUT = -5,     /* reserved: no kernel of this library waits on the device, so nothing returns it */
     HPSGD_E_UNSUPPORTED = -6  /* size beyond a documented limit */
 } hpsgd_status;
 
@@ -57,22 +57,44 @@ enum {
                                    Results do not depend on it. Default 1. */
     HPSGD_OPT_PROFILE = 6,      /* 1: bracket every kernel launch of the path with CUDA events
                                    on the stream it runs on (see hpsgd_profile_read). */
-    HPSGD_OPT_FUSE = 7          /* 1: hpsgd_sync_merge does not launch its merge at once; if the next
-                                   call is a batched local step (hpsgd_local_step_all[_ex], K <= 32)
-                                   both run as ONE kernel in which the re-cloned replica never goes
-                                   to memory; any other call first launches the merge on its own.
-                                   Same operations in the same order: results are bit-identical.
-                                   2: as 1, and additionally, when momentum != 0, K is 4, 8 or 16 and
-                                   every worker made exactly one local step since the last merge, the
-                                   replica rows are neither read nor written: the replica the previous
-                                   step stored is fma(-mu, m_i, w) of values still in memory, and that
-                                   one FMA is recomputed instead (bit-identical).  The rows are rebuilt
-                                   before anything else reads them (hpsgd_synchronize, a per-worker
-                                   step, a merge on its own, a checkpoint).  Default 0. */
+    HPSGD_OPT_FUSE = 7,         /* How a round is cut into kernels (replica-change form, K <= 32; otherwise
+                                   as 0).  Every setting performs the same operations in the same order,
+                                   so results are bit-identical.
+                                   0 (default): the paper's two processes.  Every call launches at once:
+                                      local steps on the main stream, the merge on the side stream, where it
+                                      overlaps whatever the caller does until the next local step.
+                                   1: hpsgd_sync_merge holds its merge back; if the next call is a batched
+                                      local step (hpsgd_local_step_all[_ex]) both run as ONE kernel in
+                                      which the re-cloned replicas never go to memory before they are
+                                      stepped; any other call first launches the merge on its own.
+                                   2: one kernel per round.  A batched local step is held back; the
+                                      hpsgd_sync_merge that follows runs it together with the merge: every
+                                      worker is stepped in registers, its change enters the K-way sum, and
+                                      the stepped replica is never stored, because the merge re-clones it
+                                      anyway.  Merges also stop writing the K re-cloned replicas: a replica
+                                      that nothing has stepped since its clone IS w and is read from w
+                                      ("lazy clone"; hpsgd_get_replica then returns w's address).  With one
+                                      local step per worker and period no replica row is read or written
+                                      at all: per index w, D, K momenta and K gradients come in and w, D,
+                                      K momenta go out.  Any other call first launches a held-back step on
+                                      its own.  The gradients of a held-back step are read when it is
+                                      launched: leave them alone until the next library call returns.
+                                   For callers whose gradients are already resident (a simulation, a
+                                   benchmark) 2 is the fastest; a trainer that computes the next gradients
+                                   while the merge runs wants 0. */
+    HPSGD_OPT_DEBUG_GROUP_LIMIT = 8 /* Checked build (compiled with -DHPSGD_DEBUG) only; HPSGD_E_UNSUPPORTED
+                                   otherwise.  In that build every hot kernel tests each 8-element group
+                                   index against the number of groups of a flat buffer before touching
+                                   memory; a group that fails is skipped and recorded, and the next call
+                                   that waits for the device (hpsgd_synchronize, hpsgd_get_global, ...)
+                                   returns HPSGD_E_CUDA with the record.  This option lowers the number
+                                   the kernels test against (value = groups, -1 = the real one), so that
+                                   the guard can be seen to work on accesses that are in fact in bounds. */
 };
 
 /* Kernel kinds of hpsgd_profile_read. */
-enum { HPSGD_KERNEL_LOCAL_STEP = 0, HPSGD_KERNEL_MERGE = 1, HPSGD_KERNEL_MERGE_STEP = 2 };
+enum { HPSGD_KERNEL_LOCAL_STEP = 0, HPSGD_KERNEL_MERGE = 1, HPSGD_KERNEL_MERGE_STEP = 2 /* fuse 1 */,
+       HPSGD_KERNEL_ROUND = 3 /* fuse 2: local steps + merge */ };
 
 enum { HPSGD_F32 = 0, HPSGD_BF16 = 1 };
 
@@ -217,7 +239,11 @@ int hpsgd_set_option(int key, double value);
  * aligned) their values.  Rows not listed have gradient ZERO and are still stepped
  * (momentum decays and moves the replica, weight decay applies): the result equals
  * a dense step with zero rows.  row_idx == NULL or n_rows == 0 means no sparse tensor
- * rows are active.  Unsorted, duplicate or out-of-range rows are the caller's error.
+ * rows are active.  Unsorted, duplicate or out-of-range rows are the caller's error: the
+ * normal build does not look (an out-of-range row is ignored, a duplicate leaves it open
+ * which of its values is used).  The checked build (-DHPSGD_DEBUG) copies row_idx to the
+ * host, waiting for the main stream, and returns HPSGD_E_BADARG for such a list before
+ * anything is enqueued.
  */
 typedef struct hpsgd_grad_desc {
     const void* dense;
@@ -276,6 +302,8 @@ int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs);
  *
  * The first call on each device looks up the device address of the built-in array (with
  * that device current) and remembers it; make that first call outside any stream capture.
+ * That look-up is safe against several host threads arriving together; everything else
+ * about the call follows the rule of this library: one host thread at a time.
  * All calls on one device share the one array, and it keeps whatever the previous call
  * left: each call therefore resets the entries it uses before filling them.  Two calls
  * whose GPU work can overlap (different streams without an ordering between them) race
@@ -305,6 +333,14 @@ int hpsgd_local_step_host(int worker, const void* host_grads);
  * tensors) and reset D = 0, r_i = w, m_i = 0, merge count 0.  Blocking. */
 int hpsgd_set_global_host(const float* host_w, int64_t n);
 
+/*
+ * Start again from a freshly seeded model (Algorithm 2, initialisation): `seed` replaces the
+ * seed of hpsgd_init for every hash stream, w is filled on the device with the uniform
+ * [-0.1, 0.1) values of stream 2 exactly as hpsgd_init fills it, and D = 0, r_i = w, m_i = 0,
+ * merge count 0.  Layout, K, options and schedule stay.  Blocking.
+ */
+int hpsgd_fill_global(uint64_t seed);
+
 /* Wait for all work, then copy the P parameters of w (un-padded concatenation) to a
  * HOST array of n = P floats.  Blocking. */
 int hpsgd_copy_global(float* host_out, int64_t n);
@@ -317,8 +353,9 @@ int hpsgd_copy_global_async(float* host_out, int64_t n);
 
 /* Device pointers (P_pad floats each) to worker's replica and momentum buffer (*m = NULL
  * when momentum == 0), and to the pending change D.  Any out pointer may be NULL.
- * Does not synchronise: call hpsgd_synchronize first, which also launches a deferred merge
- * and rebuilds replica rows that HPSGD_OPT_FUSE = 2 left implicit. */
+ * Does not synchronise: call hpsgd_synchronize first, which also launches whatever
+ * HPSGD_OPT_FUSE held back.  For a replica that is a lazy clone (HPSGD_OPT_FUSE = 2, the
+ * pipelined schedule) the pointer is w itself; ask again after the next local step. */
 int hpsgd_get_replica(int worker, const float** r, const float** m);
 int hpsgd_get_pending(const float** D);
 
@@ -376,14 +413,14 @@ int hpsgd_synchronize(void);
 
 /*
  * With HPSGD_OPT_PROFILE on: total device milliseconds and number of launches of one kind
- * of kernel (HPSGD_KERNEL_*: local step, merge, fused merge + local step) since the last
+ * of kernel (HPSGD_KERNEL_*: local step, merge, merge + next local step, whole round) since the last
  * read of that kind, measured with CUDA event pairs recorded around each launch on the
  * stream it ran on.  Launches any deferred merge, synchronises, and resets that kind's
  * totals.  Any out pointer may be NULL.
  */
 int hpsgd_profile_read(int kind, double* ms, int64_t* launches);
 
-/* Enqueue a merge that HPSGD_OPT_FUSE deferred, if there is one (does not wait). */
+/* Enqueue what HPSGD_OPT_FUSE held back (a merge, or a batched local step), if anything (does not wait). */
 int hpsgd_flush(void);
 
 /* Number of kernels this library has launched since hpsgd_init. */

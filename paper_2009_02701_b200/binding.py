@@ -15,7 +15,8 @@ HPSGD_E_BADARG, HPSGD_E_STATE, HPSGD_E_NOMEM = -1, -2, -3
 HPSGD_E_CUDA, HPSGD_E_TIMEOUT, HPSGD_E_UNSUPPORTED = -4, -5, -6
 HPSGD_OPT_WEIGHT_DECAY, HPSGD_OPT_STALENESS, HPSGD_OPT_GRAD_DTYPE = 1, 2, 3
 HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE, HPSGD_OPT_FUSE = 4, 5, 6, 7
-HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP = 0, 1, 2
+HPSGD_OPT_DEBUG_GROUP_LIMIT = 8
+HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP, HPSGD_KERNEL_ROUND = 0, 1, 2, 3
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
@@ -60,6 +61,7 @@ SIGNATURES = {
                                               _f32, _f32, _f32, _vp]),
     "hpsgd_local_step_host": (_ci, [_ci, _vp]),
     "hpsgd_set_global_host": (_ci, [_vp, _i64]),
+    "hpsgd_fill_global": (_ci, [_u64]),
     "hpsgd_copy_global": (_ci, [_vp, _i64]),
     "hpsgd_copy_global_async": (_ci, [_vp, _i64]),
     "hpsgd_get_replica": (_ci, [_ci, _P(_vp), _P(_vp)]),
@@ -80,6 +82,14 @@ SIGNATURES = {
 }
 
 _lib = None
+
+
+def use_library(path=None):
+    """Point the binding at another build of the library (the checked build, say); None = the
+    in-tree one.  Call hpsgd_destroy() first: each loaded library has its own state."""
+    global _lib, LIB_PATH
+    _lib = None
+    LIB_PATH = os.path.join(HERE, "libhpsgd.so") if path is None else str(path)
 
 
 def load():
@@ -225,6 +235,10 @@ def _count(x):
 
 def hpsgd_set_global_host(host_w):
     return _check(load().hpsgd_set_global_host(_ptr(host_w), _count(host_w)))
+
+
+def hpsgd_fill_global(seed):
+    return _check(load().hpsgd_fill_global(int(seed)))
 
 
 def hpsgd_copy_global(host_out):

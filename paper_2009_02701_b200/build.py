@@ -25,22 +25,28 @@ def nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; returns its path."""
-    if not force and os.path.exists(LIB):
+def build(force: bool = False, verbose: bool = False, debug: bool = False, out: str | None = None) -> str:
+    """Compile the library if it is missing or older than its sources; returns its path.
+
+    ``debug`` builds the checked variant (-DHPSGD_DEBUG: kernel guards that record and skip an
+    out-of-range access, host-side validation of sparse row lists) into ``out`` (default
+    ``libhpsgd_debug.so`` beside the normal library)."""
+    lib = out or (os.path.join(HERE, "libhpsgd_debug.so") if debug else LIB)
+    if not force and os.path.exists(lib):
         newest = max(os.path.getmtime(p) for p in DEPENDS)
-        if os.path.getmtime(LIB) >= newest:
-            return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
+        if os.path.getmtime(lib) >= newest:
+            return lib
+    tmp = lib + ".tmp.%d" % os.getpid()
+    cmd = [nvcc(), *NVCC_FLAGS, *(["-DHPSGD_DEBUG"] if debug else []), *(["-Xptxas", "-v"] if verbose else []),
+           "-o", tmp, *SOURCES]
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n%s\n%s" % (proc.stdout, proc.stderr))
     if verbose:
         sys.stderr.write(proc.stderr)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

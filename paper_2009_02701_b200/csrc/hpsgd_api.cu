@@ -148,7 +148,8 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.r = reinterpret_cast<float*>(g.arena + a.r);
     g.m = mom ? reinterpret_cast<float*>(g.arena + a.m) : nullptr;
     g.d_table = reinterpret_cast<int64_t*>(g.arena + a.table);
-    g.steps_in_period.assign(K, 0);
+    g.at_w.assign(K, 1);
+    g.row_valid.assign(K, 1);
     g.wbuf[0] = g.w;
     g.rbuf[0] = g.r;
     if (g.pipeline) {
@@ -213,7 +214,6 @@ int hpsgd_synchronize(void)
 {
     TRY(need_init());
     TRY(flush_deferred());
-    TRY(ensure_replicas());
     TRY(sync_all());
     return check_async();
 }
@@ -256,7 +256,17 @@ int hpsgd_set_option(int key, double value)
     case HPSGD_OPT_FUSE:
         if (value != 0.0 && value != 1.0 && value != 2.0) return fail(HPSGD_E_BADARG, "fuse must be 0, 1 or 2");
         g.fuse = (int)value;
+        if (!lazy_clones() && !g.pipeline) TRY(materialize_clones());   // the other schedules read replica rows
         return HPSGD_OK;
+    case HPSGD_OPT_DEBUG_GROUP_LIMIT:
+#ifdef HPSGD_DEBUG
+        if (!(value >= -1.0 && value <= (double)(g.P_pad / 8) && value == (double)(int64_t)value))
+            return fail(HPSGD_E_BADARG, "the limit must be -1 (the real one) or a whole number of groups in [0, P_pad / 8]");
+        g.debug_limit = (int64_t)value;
+        return HPSGD_OK;
+#else
+        return fail(HPSGD_E_UNSUPPORTED, "only the checked build (HPSGD_DEBUG) has kernel guards");
+#endif
     case HPSGD_OPT_PROFILE:
         if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "profile must be 0 or 1");
         TRY(prof_resolve());
@@ -307,6 +317,55 @@ int hpsgd_set_sparse_segment(int tensor_id, int64_t rows, int64_t cols)
 }
 
 // ------------------------------------------------------------------------- local steps
+}  // extern "C"
+
+namespace {
+
+// Copy stream, two staging buffers and their events of hpsgd_local_step_host: built into locals
+// and handed to the state only when all of it exists, so that a failure half-way leaves nothing
+// behind and the next call simply tries again.
+int make_host_staging()
+{
+    cudaStream_t copy = nullptr;
+    void* stage[2] = {nullptr, nullptr};
+    cudaEvent_t copied[2] = {nullptr, nullptr}, freed[2] = {nullptr, nullptr};
+    int rc = HPSGD_OK;
+    cudaError_t e = cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking);
+    if (e != cudaSuccess) rc = fail(HPSGD_E_CUDA, "could not create the copy stream: %s", cudaGetErrorString(e));
+    for (int b = 0; b < 2 && rc == HPSGD_OK; ++b) {
+        e = cudaMalloc(&stage[b], (size_t)g.P_pad * 4);
+        if (e != cudaSuccess) {
+            rc = fail(HPSGD_E_NOMEM, "cudaMalloc of the staging buffer failed: %s", cudaGetErrorString(e));
+            break;
+        }
+        e = cudaEventCreateWithFlags(&copied[b], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&freed[b], cudaEventDisableTiming);
+        if (e != cudaSuccess) rc = fail(HPSGD_E_CUDA, "could not create the staging events: %s", cudaGetErrorString(e));
+    }
+    if (rc != HPSGD_OK) {
+        for (int b = 0; b < 2; ++b) {
+            if (stage[b]) cudaFree(stage[b]);
+            if (copied[b]) cudaEventDestroy(copied[b]);
+            if (freed[b]) cudaEventDestroy(freed[b]);
+        }
+        if (copy) cudaStreamDestroy(copy);
+        cudaGetLastError();
+        return rc;
+    }
+    for (int b = 0; b < 2; ++b) {
+        g.stage[b] = stage[b];
+        g.stage_copied[b] = copied[b];
+        g.stage_free[b] = freed[b];
+        g.stage_used[b] = false;
+    }
+    g.copy = copy;
+    return HPSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 int hpsgd_local_step(int worker, const void* grads)
 {
     TRY(need_init());
@@ -324,6 +383,7 @@ int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc)
     TRY(check_worker(worker));
     if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
     TRY(check_desc(desc));
+    TRY(validate_rows(desc, g.sp_rows, g.main));
     TRY(flush_deferred());
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(worker, 1, desc, &gp));
@@ -343,6 +403,14 @@ int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes)
         return enqueue_fused(gp, false);
     }
     TRY(flush_deferred());
+    if (lazy_clones()) {                   // fuse 2: held back for the merge it will run with
+        g.deferred_gp = BatchPtrs{};
+        for (int i = 0; i < g.K; ++i)
+            g.deferred_gp.dense[i] = static_cast<const char*>(grads) + (int64_t)i * worker_stride_bytes;
+        g.deferred_sparse = false;
+        g.step_deferred = true;
+        return HPSGD_OK;
+    }
     for (int w0 = 0; w0 < g.K; w0 += kMaxBatch) {
         const int nw = std::min(kMaxBatch, g.K - w0);
         BatchPtrs gp{};
@@ -359,9 +427,17 @@ int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs)
     if (g.K > kMaxBatch) return fail(HPSGD_E_UNSUPPORTED, "batched sparse steps support K <= %d", kMaxBatch);
     if (!descs) return fail(HPSGD_E_BADARG, "descriptor array is NULL");
     for (int i = 0; i < g.K; ++i) TRY(check_desc(descs + i));
+    for (int i = 0; i < g.K; ++i) TRY(validate_rows(descs + i, g.sp_rows, g.main));
+    if (g.step_deferred) TRY(flush_deferred());          // an earlier held-back step still uses the slot maps
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(0, g.K, descs, &gp));
     if (g.merge_deferred) return enqueue_fused(gp, true);
+    if (lazy_clones()) {
+        g.deferred_gp = gp;
+        g.deferred_sparse = true;
+        g.step_deferred = true;
+        return HPSGD_OK;
+    }
     return enqueue_local(0, g.K, gp, true);
 }
 
@@ -372,18 +448,7 @@ int hpsgd_local_step_host(int worker, const void* host_grads)
     if (!host_grads) return fail(HPSGD_E_BADARG, "host_grads is NULL");
     TRY(flush_deferred());
     const size_t bytes = (size_t)g.P_pad * (g.grad_dtype == HPSGD_BF16 ? 2 : 4);
-    if (!g.copy) {
-        CUDA_TRY(cudaStreamCreateWithFlags(&g.copy, cudaStreamNonBlocking));
-        for (int b = 0; b < 2; ++b) {
-            cudaError_t e = cudaMalloc(&g.stage[b], (size_t)g.P_pad * 4);
-            if (e != cudaSuccess) {
-                cudaGetLastError();
-                return fail(HPSGD_E_NOMEM, "cudaMalloc of the staging buffer failed: %s", cudaGetErrorString(e));
-            }
-            CUDA_TRY(cudaEventCreateWithFlags(&g.stage_copied[b], cudaEventDisableTiming));
-            CUDA_TRY(cudaEventCreateWithFlags(&g.stage_free[b], cudaEventDisableTiming));
-        }
-    }
+    if (!g.copy) TRY(make_host_staging());
     const int b = g.stage_next;
     g.stage_next ^= 1;
     if (g.stage_used[b]) CUDA_TRY(cudaStreamWaitEvent(g.copy, g.stage_free[b], 0));
@@ -402,20 +467,15 @@ int hpsgd_local_step_host(int worker, const void* host_grads)
 int hpsgd_sync_merge(void)
 {
     TRY(need_init());
-    TRY(flush_deferred());                 // two merges in a row: the earlier one runs on its own
+    if (g.merge_deferred) TRY(flush_deferred());   // two merges in a row: the earlier one runs on its own
     int flags = 0;
     if (g.staleness == 0) flags |= kMergeImmediate;
     else if (g.D_valid) flags |= kMergeApplyPending;
     g.D_valid = true;
     g.merges += 1;
-    bool all_single = true;
-    for (int& n : g.steps_in_period) {
-        all_single = all_single && n == 1;
-        n = 0;
-    }
-    g.deferred_all_single = all_single;
+    if (g.step_deferred) return enqueue_round(flags);    // fuse 2: the held-back step and this merge, one kernel
     if (g.pipeline) return enqueue_pipelined_merge(flags);
-    if (g.fuse && g.form == HPSGD_FORM_REPLICA_CHANGE) {
+    if (g.fuse == 1 && g.form == HPSGD_FORM_REPLICA_CHANGE) {
         g.merge_deferred = true;
         g.deferred_flags = flags;
         return HPSGD_OK;
@@ -449,6 +509,23 @@ int hpsgd_set_global_host(const float* host_w, int64_t n)
     for (size_t t = 0; t < g.sizes.size(); ++t)
         CUDA_TRY(cudaMemcpyAsync(g.w + g.offsets[t], host_w + g.starts[t], (size_t)g.sizes[t] * 4,
                                  cudaMemcpyHostToDevice, g.main));
+    return reset_state_from_w();
+}
+
+int hpsgd_fill_global(uint64_t seed)
+{
+    TRY(need_init());
+    TRY(flush_deferred());
+    TRY(sync_all());
+    g.seed = seed;
+    g.key = mix64(seed + kM3);
+    const size_t n = g.sizes.size();
+    CUDA_TRY(cudaMemsetAsync(g.w, 0, (size_t)g.stride * 4, g.main));
+    const GenParams gp = gen_params(0, 0, 2, 0.0);
+    gen_flat_kernel<false><<<grid_for(gen_flat_kernel<false>, g.P_pad, kThreads), kThreads, 0, g.main>>>(
+        g.w, g.P_pad, g.d_table, g.d_table + n, g.d_table + 2 * n, (int)n, gp);
+    ++g.launches;
+    TRY(check_async());
     return reset_state_from_w();
 }
 
@@ -493,7 +570,7 @@ int hpsgd_get_replica(int worker, const float** r, const float** m)
 {
     TRY(need_init());
     TRY(check_worker(worker));
-    if (r) *r = (g.pipeline && !g.touched[worker]) ? g.w : g.r + (int64_t)worker * g.stride;
+    if (r) *r = g.pipeline ? (g.touched[worker] ? g.r + (int64_t)worker * g.stride : g.w) : replica_src(worker);
     if (m) *m = g.m ? g.m + (int64_t)worker * g.stride : nullptr;
     return HPSGD_OK;
 }
@@ -534,7 +611,6 @@ int hpsgd_export_state(void* host_out, size_t bytes)
     TRY(need_init());
     if (!host_out || bytes < state_bytes()) return fail(HPSGD_E_BADARG, "need a host buffer of hpsgd_state_bytes() = %zu bytes", state_bytes());
     TRY(flush_deferred());
-    TRY(ensure_replicas());
     TRY(sync_all());
     StateHeader h{};
     h.magic = kStateMagic;
@@ -547,8 +623,8 @@ int hpsgd_export_state(void* host_out, size_t bytes)
     CUDA_TRY(cudaMemcpy(out, g.w, row, cudaMemcpyDeviceToHost)); out += row;
     CUDA_TRY(cudaMemcpy(out, g.D, row, cudaMemcpyDeviceToHost)); out += row;
     for (int i = 0; i < g.K; ++i) {
-        // pipelined schedule: a worker that has not stepped since the last synchronisation has w as its replica
-        const float* src = (g.pipeline && !g.touched[i]) ? g.w : g.r + (int64_t)i * g.stride;
+        // a worker that has not stepped since the last synchronisation may have w itself as its replica
+        const float* src = g.pipeline ? (g.touched[i] ? g.r + (int64_t)i * g.stride : g.w) : replica_src(i);
         CUDA_TRY(cudaMemcpy(out, src, row, cudaMemcpyDeviceToHost)); out += row;
     }
     if (g.m)
@@ -568,6 +644,9 @@ int hpsgd_import_state(const void* host_in, size_t bytes)
     if (h.P != g.P || h.P_pad != g.P_pad || h.K != g.K || h.form != g.form || h.has_aux != (g.m ? 1 : 0))
         return fail(HPSGD_E_BADARG, "state blob does not match the initialised sizes, form or optimiser");
     if (bytes < state_bytes()) return fail(HPSGD_E_BADARG, "state blob truncated");
+    if (h.staleness != 0 && h.staleness != 1) return fail(HPSGD_E_BADARG, "state blob holds staleness %d", h.staleness);
+    if (g.pipeline && h.staleness != 1)
+        return fail(HPSGD_E_BADARG, "the pipelined schedule needs the one-synchronisation delay; the blob was written with staleness 0");
     if (h.staleness != g.staleness && g.merges) return fail(HPSGD_E_STATE, "staleness differs and merges have already run");
     TRY(flush_deferred());
     TRY(sync_all());
@@ -586,8 +665,8 @@ int hpsgd_import_state(const void* host_in, size_t bytes)
     g.D_valid = h.D_valid != 0;
     g.merges = h.merges;
     if (g.pipeline) std::fill(g.touched.begin(), g.touched.end(), 1);   // every replica row now holds real data
-    g.replicas_stale = false;
-    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 2);   // unknown history: not "exactly one step"
+    std::fill(g.row_valid.begin(), g.row_valid.end(), 1);
+    std::fill(g.at_w.begin(), g.at_w.end(), 0);                         // unknown history: the rows are what counts
     g.reduce_outstanding = false;
     std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
     std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
@@ -615,6 +694,7 @@ int64_t hpsgd_tensor_offset(int tensor_id)
 int hpsgd_gen_grads(void* out, int worker, int step, int kind, double scale)
 {
     TRY(check_gen_args(out, worker, step, kind));
+    if (g.step_deferred) TRY(flush_deferred());   // a held-back step may still have to read what `out` holds now
     const GenParams gp = gen_params(worker, step, kind, scale);
     const size_t n = g.sizes.size();
     if (g.grad_dtype == HPSGD_BF16)
@@ -635,6 +715,7 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
     if (n_rows < 0 || n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows out of range");
     if (n_rows == 0) return HPSGD_OK;
     if (!row_idx) return fail(HPSGD_E_BADARG, "row_idx is NULL");
+    if (g.step_deferred) TRY(flush_deferred());
     const GenParams gp = gen_params(worker, step, kind, scale);
     const int64_t n = (int64_t)n_rows * g.sp_cols;
     if (g.grad_dtype == HPSGD_BF16)
@@ -649,7 +730,7 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
 int hpsgd_profile_read(int kind, double* ms, int64_t* launches)
 {
     TRY(need_init());
-    if (kind < 0 || kind > 2) return fail(HPSGD_E_BADARG, "unknown kernel kind %d", kind);
+    if (kind < 0 || kind > 3) return fail(HPSGD_E_BADARG, "unknown kernel kind %d", kind);
     TRY(flush_deferred());
     TRY(sync_all());
     TRY(prof_resolve());
@@ -674,40 +755,35 @@ namespace {
 
 constexpr int kNoallocMaxDevices = 64;
 struct NoallocDevice {
-    bool ready = false;
+    std::once_flag once;
+    cudaError_t status = cudaErrorUnknown;
     int32_t* slot = nullptr;     // device address of g_noalloc_slot on this device
-    int sm_count = 0;
 } g_noalloc_dev[kNoallocMaxDevices];
 
 // Once per device, with that device current: g_noalloc_slot names a host-side stand-in in
-// host code, so the address a kernel can use has to be asked for.
-int noalloc_setup(int dev, NoallocDevice** out)
+// host code, so the address a kernel can use has to be asked for.  std::call_once makes the
+// look-up safe when several host threads make their first call on a device together.
+int noalloc_setup(int dev, int32_t** slot)
 {
     if (dev < 0 || dev >= kNoallocMaxDevices) return fail(HPSGD_E_UNSUPPORTED, "device index %d not supported", dev);
     NoallocDevice& d = g_noalloc_dev[dev];
-    if (!d.ready) {
+    std::call_once(d.once, [&d] {
         void* p = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_slot);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            return fail(HPSGD_E_CUDA, "cudaGetSymbolAddress of the scratch map failed: %s", cudaGetErrorString(e));
-        }
-        int sms = 0;
-        CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        d.slot = static_cast<int32_t*>(p);
-        d.sm_count = sms;
-        d.ready = true;
-    }
-    *out = &d;
+        d.status = cudaGetSymbolAddress(&p, g_noalloc_slot);
+        if (d.status == cudaSuccess) d.slot = static_cast<int32_t*>(p);
+        else cudaGetLastError();
+    });
+    if (d.status != cudaSuccess)
+        return fail(HPSGD_E_CUDA, "cudaGetSymbolAddress of the scratch map failed: %s", cudaGetErrorString(d.status));
+    *slot = d.slot;
     return HPSGD_OK;
 }
 
 template <bool BF16, bool MOM, bool WD>
-void noalloc_launch(cudaStream_t s, int sm_count, float* r, float* m, const BatchPtrs& gp,
-                    const SparseSeg& seg, int64_t n, const StepParams& p)
+void noalloc_launch(cudaStream_t s, float* r, float* m, const BatchPtrs& gp, const SparseSeg& seg, int64_t n,
+                    const StepParams& p)
 {
-    (void)sm_count;
-    local_step_kernel<BF16, MOM, WD, true><<<hot_grid(n), kHotThreads, 0, s>>>(r, m, 0, 0, gp, seg, 0, n, p);
+    local_step_kernel<BF16, MOM, WD, true><<<hot_grid(n), kHotThreads, 0, s>>>(r, m, 0, 0, gp, seg, 0, n, p, n);
 }
 
 }  // namespace
@@ -728,7 +804,8 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
     if (rows > HPSGD_NOALLOC_MAX_ROWS)
         return fail(HPSGD_E_UNSUPPORTED, "%lld rows exceed the built-in scratch map of %d rows; use hpsgd_local_step_ex",
                     (long long)rows, HPSGD_NOALLOC_MAX_ROWS);
-    if (seg_offset < 0 || seg_offset % 8 || seg_offset + rows * cols > n_elems)
+    // tested by division first, so that rows * cols is only formed when it cannot overflow
+    if (cols > n_elems || rows > n_elems / cols || seg_offset < 0 || seg_offset % 8 || seg_offset > n_elems - rows * cols)
         return fail(HPSGD_E_BADARG, "the sparse tensor does not fit inside the flat buffer");
     if (!desc) return fail(HPSGD_E_BADARG, "descriptor is NULL");
     TRY(check_grad_ptr(desc->dense, "dense gradient"));
@@ -738,15 +815,16 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
 
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
-    NoallocDevice* d = nullptr;
-    TRY(noalloc_setup(dev, &d));
+    int32_t* slot = nullptr;
+    TRY(noalloc_setup(dev, &slot));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TRY(validate_rows(desc, rows, s));     // checked build only
 
     // the map keeps the previous call's contents: every row starts again at "no slot" (-1)
-    CUDA_TRY(cudaMemsetAsync(d->slot, 0xFF, (size_t)rows * 4, s));
+    CUDA_TRY(cudaMemsetAsync(slot, 0xFF, (size_t)rows * 4, s));
     if (have_rows) {
         SlotBatch sb{};
-        sb.slot[0] = d->slot;
+        sb.slot[0] = slot;
         sb.row_idx[0] = desc->row_idx;
         sb.n_rows[0] = desc->n_rows;
         scatter_slots_kernel<<<dim3((desc->n_rows + 255) / 256, 1), 256, 0, s>>>(sb, rows);
@@ -754,12 +832,13 @@ extern "C" int hpsgd_local_step_sparse_noalloc(float* replica, float* momentum_b
     BatchPtrs gp{};
     gp.dense[0] = desc->dense;
     gp.row_vals[0] = desc->row_vals;
-    gp.slot[0] = d->slot;
+    gp.slot[0] = slot;
+    gp.n_rows[0] = have_rows ? desc->n_rows : 0;
     SparseSeg seg{seg_offset / 8, (seg_offset + rows * cols) / 8, (int32_t)(cols / 8)};
     const StepParams p{-lr, momentum, weight_decay};
     const bool mom = momentum != 0.f, wd = weight_decay != 0.f, bf = grad_dtype == HPSGD_BF16;
     const int64_t nvec = n_elems / 8;
-#define HPSGD_NOALLOC_CASE(B, M, W) noalloc_launch<B, M, W>(s, d->sm_count, replica, momentum_buf, gp, seg, nvec, p)
+#define HPSGD_NOALLOC_CASE(B, M, W) noalloc_launch<B, M, W>(s, replica, momentum_buf, gp, seg, nvec, p)
     if (bf) {
         if (mom && wd) HPSGD_NOALLOC_CASE(true, true, true);
         else if (mom) HPSGD_NOALLOC_CASE(true, true, false);

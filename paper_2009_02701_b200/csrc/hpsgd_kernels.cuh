@@ -21,6 +21,45 @@ namespace hpsgd {
 constexpr int kThreads = 256;      // support kernels (generators, clone)
 constexpr int kHotThreads = 128;   // local step and merge: one 8-element group per thread
 
+// ---------------------------------------------------------------------------- checked build
+// Compiled with -DHPSGD_DEBUG every hot kernel tests the group index it is about to touch
+// against the number of groups of a flat buffer (and a row -> slot entry against the number
+// of rows it may name) before any access.  A violation is recorded in g_debug_report (first
+// one wins) and that group is skipped: nothing traps, nothing waits, the context stays
+// usable, and the host turns the record into an error at its next synchronisation.  In the
+// normal build the guards compile to nothing.
+enum KernelId { kIdLocalStep = 1, kIdMerge, kIdMergeLazy, kIdMergeStep, kIdRound, kIdCommit, kIdReduce,
+                kIdAccumStep, kIdAccumMerge, kIdScatter };
+
+#ifdef HPSGD_DEBUG
+struct DebugReport {
+    int code;            // 0: nothing recorded; 1: group index out of range; 2: slot out of range; 3: row out of range
+    int kernel;          // KernelId
+    long long index;     // the offending group / slot / row
+    long long limit;     // what it was tested against
+};
+__device__ DebugReport g_debug_report;
+
+__device__ __forceinline__ bool debug_check(bool ok, int code, int kernel, long long index, long long limit)
+{
+    if (ok) return true;
+    if (atomicCAS(&g_debug_report.code, 0, code) == 0) {
+        g_debug_report.kernel = kernel;
+        g_debug_report.index = index;
+        g_debug_report.limit = limit;
+    }
+    return false;
+}
+#define HPSGD_GUARD_GROUP(o, limit, kernel) \
+    if (!hpsgd::debug_check((o) >= 0 && (o) < (limit), 1, (kernel), (long long)(o), (long long)(limit))) continue
+#define HPSGD_SLOT_OK(s, n_rows, kernel) hpsgd::debug_check((s) < (n_rows), 2, (kernel), (long long)(s), (long long)(n_rows))
+#define HPSGD_ROW_OK(row, rows, kernel) hpsgd::debug_check((row) >= 0 && (row) < (rows), 3, (kernel), (long long)(row), (long long)(rows))
+#else
+#define HPSGD_GUARD_GROUP(o, limit, kernel) do { } while (0)
+#define HPSGD_SLOT_OK(s, n_rows, kernel) true
+#define HPSGD_ROW_OK(row, rows, kernel) ((row) >= 0 && (row) < (rows))
+#endif
+
 // ---------------------------------------------------------------------------- memory ops
 // The hot kernels move 8 consecutive fp32 values (32 bytes) per thread with the 256-bit
 // global loads/stores of sm_100 (ld/st.global.v8.b32); addresses are 32-byte aligned.
@@ -146,9 +185,10 @@ struct BatchPtrs {
     const void* dense[kMaxBatch];
     const void* row_vals[kMaxBatch];
     const int32_t* slot[kMaxBatch];
+    int32_t n_rows[kMaxBatch];       // rows listed for the sparse-row tensor (what a slot may name)
     const float* r_src[kMaxBatch];   // where the worker's replica is READ from; NULL: its own row.
-                                     // (pipelined schedule: the first step after a synchronisation
-                                     // reads the global model, which is the not-yet-written clone)
+                                     // (a replica that is still the clone of the global model is
+                                     // read from w itself when its row has not been written)
 };
 
 // One worker per blockIdx.y; workers' replicas/momenta are `stride` floats apart starting
@@ -158,9 +198,9 @@ struct BatchPtrs {
 // about 10 % faster than one resident wave striding through memory); the loop only
 // matters when n exceeds what a grid can index.
 template <bool BF16, bool MOM, bool WD, bool SPARSE>
-__global__ void __launch_bounds__(kHotThreads)
+__global__ void __launch_bounds__(kHotThreads, 8)
 local_step_kernel(float* __restrict__ r_base, float* __restrict__ m_base, int64_t stride,
-                  int w0, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, StepParams p)
+                  int w0, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, StepParams p, int64_t lim)
 {
     const int wk = blockIdx.y;
     float* __restrict__ r = r_base + (int64_t)(w0 + wk) * stride;
@@ -172,6 +212,7 @@ local_step_kernel(float* __restrict__ r_base, float* __restrict__ m_base, int64_
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     const float* __restrict__ rs = gp.r_src[wk] ? gp.r_src[wk] : r;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdLocalStep);
         f8 rr = ld8(rs + o * 8);
         f8 mm;
         if (MOM) mm = ld8(m + o * 8);
@@ -183,7 +224,8 @@ local_step_kernel(float* __restrict__ r_base, float* __restrict__ m_base, int64_
                 const int64_t rel = o - seg.o_begin;
                 const int64_t row = rel / seg.cols8;
                 const int32_t s = __ldg(slot + row);
-                if (s >= 0) gg = load_grad8<BF16>(rv, (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
+                if (s >= 0 && HPSGD_SLOT_OK(s, gp.n_rows[wk], kIdLocalStep))
+                    gg = load_grad8<BF16>(rv, (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
                 else gg = zero8();
             }
         }
@@ -209,7 +251,7 @@ __global__ void scatter_slots_kernel(SlotBatch sb, int64_t rows)
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k < sb.n_rows[i]) {
         const int32_t row = sb.row_idx[i][k];
-        if (row >= 0 && row < rows) sb.slot[i][row] = k;
+        if (HPSGD_ROW_OK(row, rows, kIdScatter)) sb.slot[i][row] = k;
     }
 }
 
@@ -269,11 +311,12 @@ constexpr int kMergeImmediate = 2;      // flags: staleness 0
 template <int KT>
 __global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
 merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r, int64_t stride,
-             int K, int64_t o0, int64_t n, int flags)
+             int K, int64_t o0, int64_t n, int flags, int64_t lim)
 {
     const float fK = (float)K;
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdMerge);
         const int64_t e = o * 8;
         const f8 wv = ld8(w + e);
         f8 dv = zero8();
@@ -319,10 +362,11 @@ merge_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r
 // touch different memory.  Same operations and order as merge_kernel.
 __global__ void __launch_bounds__(kHotThreads)
 commit_kernel(const float* __restrict__ w, const float* __restrict__ D, float* __restrict__ w_next,
-              int64_t n, int flags)
+              int64_t n, int flags, int64_t lim)
 {
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdCommit);
         f8 wv = ld8(w + o * 8);
         if (flags & kMergeApplyPending) {
             const f8 dv = ld8(D + o * 8);
@@ -333,58 +377,102 @@ commit_kernel(const float* __restrict__ w, const float* __restrict__ D, float* _
     }
 }
 
-// Per-worker source of the reduce: the worker's replica, or w itself for a worker that made
-// no local step in the period (its change is r - w = 0).
+// Per-worker source of a K-way sum: the worker's replica row, or w itself for a worker whose
+// replica is still the clone of w (it made no local step; its change is r - w = 0).
 struct ReducePtrs {
     const float* src[kMaxBatch];
 };
 
+// acc = (src_0 - w) + (src_1 - w) + ... + (src_{K-1} - w), left to right.  KT > 0: all K groups
+// are requested before the first use; KT == 0: any K, four in flight at a time.
+template <int KT>
+__device__ __forceinline__ void sum_changes_from(f8& acc, const ReducePtrs& rp, int K, int64_t e, const f8& wv)
+{
+    if constexpr (KT > 0) {
+        f8 rv[KT];
+#pragma unroll
+        for (int i = 0; i < KT; ++i) rv[i] = ld8(rp.src[i] + e);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(rv[0].v[q], wv.v[q]);
+#pragma unroll
+        for (int i = 1; i < KT; ++i)
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
+    } else {
+        {
+            const f8 r0 = ld8(rp.src[0] + e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
+        }
+        int i = 1;
+        for (; i + 4 <= K; i += 4) {
+            f8 rv[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) rv[b] = ld8(rp.src[i + b] + e);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
+        }
+        for (; i < K; ++i) {
+            const f8 ri = ld8(rp.src[i] + e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
+        }
+    }
+}
+
 template <int KT>
 __global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
-reduce_kernel(const float* __restrict__ w, float* __restrict__ D, ReducePtrs rp, int K, int64_t n)
+reduce_kernel(const float* __restrict__ w, float* __restrict__ D, ReducePtrs rp, int K, int64_t n, int64_t lim)
 {
     const int Kn = KT > 0 ? KT : K;
     const float fK = (float)Kn;
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdReduce);
         const int64_t e = o * 8;
         const f8 wv = ld8(w + e);
         f8 acc;
-        if constexpr (KT > 0) {
-            f8 rv[KT];
-#pragma unroll
-            for (int i = 0; i < KT; ++i) rv[i] = ld8(rp.src[i] + e);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(rv[0].v[q], wv.v[q]);
-#pragma unroll
-            for (int i = 1; i < KT; ++i)
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[i].v[q], wv.v[q]));
-        } else {
-            {
-                const f8 r0 = ld8(rp.src[0] + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(r0.v[q], wv.v[q]);
-            }
-            int i = 1;
-            for (; i + 4 <= K; i += 4) {
-                f8 rv[4];
-#pragma unroll
-                for (int b = 0; b < 4; ++b) rv[b] = ld8(rp.src[i + b] + e);
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(rv[b].v[q], wv.v[q]));
-            }
-            for (; i < K; ++i) {
-                const f8 ri = ld8(rp.src[i] + e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(ri.v[q], wv.v[q]));
-            }
-        }
+        sum_changes_from<KT>(acc, rp, Kn, e, wv);
         f8 dnew;
 #pragma unroll
         for (int q = 0; q < 8; ++q) dnew.v[q] = __fdiv_rn(acc.v[q], fK);
+        st8(D + e, dnew);
+    }
+}
+
+// ---------------------------------------------------------------------------- merge with a lazy clone
+// The merge without its K replica writes: after it every replica IS w, and whoever reads
+// replica i next (a local step, the next merge, an inspection call) reads w instead of a row
+// that was never written.  Same operations in the same order as merge_kernel; per index it
+// moves (K + 2) * 4 bytes in and 8 out instead of (2K + 4) * 4.  A worker whose replica is
+// already such a clone has src = w.
+template <int KT>
+__global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
+merge_lazy_kernel(float* __restrict__ w, float* __restrict__ D, ReducePtrs rp, int K, int64_t o0, int64_t n,
+                  int flags, int64_t lim)
+{
+    const int Kn = KT > 0 ? KT : K;
+    const float fK = (float)Kn;
+    const int64_t step = (int64_t)gridDim.x * kHotThreads;
+    for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdMergeLazy);
+        const int64_t e = o * 8;
+        const f8 wv = ld8(w + e);
+        f8 dv = zero8();
+        if (flags & kMergeApplyPending) dv = ld8(D + e);
+        f8 acc;
+        sum_changes_from<KT>(acc, rp, Kn, e, wv);
+        f8 dnew, wn;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            dnew.v[q] = __fdiv_rn(acc.v[q], fK);
+            wn.v[q] = wv.v[q];
+            if (flags & kMergeImmediate) wn.v[q] = __fadd_rn(wv.v[q], dnew.v[q]);
+            else if (flags & kMergeApplyPending) wn.v[q] = __fadd_rn(wv.v[q], dv.v[q]);
+        }
+        st8(w + e, wn);
         st8(D + e, dnew);
     }
 }
@@ -398,13 +486,14 @@ reduce_kernel(const float* __restrict__ w, float* __restrict__ D, ReducePtrs rp,
 template <bool BF16, bool SPARSE>
 __global__ void __launch_bounds__(kHotThreads)
 accum_step_kernel(float* __restrict__ r_base, float* __restrict__ a_base, int64_t stride,
-                  int w0, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, float neg_mu)
+                  int w0, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, float neg_mu, int64_t lim)
 {
     const int wk = blockIdx.y;
     float* __restrict__ r = r_base + (int64_t)(w0 + wk) * stride;
     float* __restrict__ a = a_base + (int64_t)(w0 + wk) * stride;
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdAccumStep);
         f8 rr = ld8(r + o * 8);
         f8 aa = ld8(a + o * 8);
         GradRaw<BF16> raw;
@@ -415,7 +504,8 @@ accum_step_kernel(float* __restrict__ r_base, float* __restrict__ a_base, int64_
                 const int64_t rel = o - seg.o_begin;
                 const int64_t row = rel / seg.cols8;
                 const int32_t s = __ldg(gp.slot[wk] + row);
-                if (s >= 0) raw = load_grad_raw<BF16>(gp.row_vals[wk], (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
+                if (s >= 0 && HPSGD_SLOT_OK(s, gp.n_rows[wk], kIdAccumStep))
+                    raw = load_grad_raw<BF16>(gp.row_vals[wk], (int64_t)s * seg.cols8 + (rel - row * seg.cols8));
                 else raw = zero_grad_raw<BF16>();
             }
         }
@@ -434,13 +524,14 @@ accum_step_kernel(float* __restrict__ r_base, float* __restrict__ a_base, int64_
 template <int KT>
 __global__ void __launch_bounds__(kHotThreads, (KT > 8 || KT == 0) ? 2 : 4)
 accum_merge_kernel(float* __restrict__ w, float* __restrict__ ghat, float* __restrict__ r, float* __restrict__ a,
-                   int64_t stride, int K, int64_t o0, int64_t n, int flags, float neg_mu)
+                   int64_t stride, int K, int64_t o0, int64_t n, int flags, float neg_mu, int64_t lim)
 {
     const int Kn = KT > 0 ? KT : K;
     const float fK = (float)Kn;
     const f8 zero = zero8();
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdAccumMerge);
         const int64_t e = o * 8;
         const f8 wv = ld8(w + e);
         f8 gv = zero;
@@ -524,7 +615,7 @@ __device__ __forceinline__ GradRaw<BF16> fused_grad_raw(const BatchPtrs& gp, con
                                                         int32_t s, int i, int64_t o)
 {
     if (SPARSE && sp.inside) {
-        if (s < 0) return zero_grad_raw<BF16>();
+        if (s < 0 || !HPSGD_SLOT_OK(s, gp.n_rows[i], kIdRound)) return zero_grad_raw<BF16>();
         return load_grad_raw<BF16>(gp.row_vals[i], (int64_t)s * seg.cols8 + sp.col8);
     }
     return load_grad_raw<BF16>(gp.dense[i], o);
@@ -534,13 +625,14 @@ template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
 __global__ void __launch_bounds__(kHotThreads, 2)
 merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r, float* __restrict__ m,
                   int64_t stride, int K, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags,
-                  StepParams p)
+                  StepParams p, int64_t lim)
 {
     constexpr int B = 4;                         // workers whose g / m are in flight together
     const int Kn = KT > 0 ? KT : K;
     const float fK = (float)Kn;
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdMergeStep);
         const int64_t e = o * 8;
         // every worker's row -> slot entry is requested up front, so that the gradient loads
         // of the step phase do not wait on a dependent lookup
@@ -623,54 +715,89 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
     }
 }
 
-// ---------------------------------------------------------------------------- merge + next local step, implicit replicas
-// With momentum and exactly one local step per worker since the last clone, the replica is
-// a function of state that is kept anyway: the step computed r_i = fma(-mu, m_i, w) from the
-// clone w and the new momentum m_i, both still in memory unchanged.  Recomputing that one FMA
-// gives the stored value bit for bit, so the replica rows need be neither read nor written:
-// per index the kernel moves (w + D + K m + K g) in and (w + D + K m) out, (3K + 4) * 4 bytes
-// with fp32 gradients instead of (5K + 4) * 4.  The replica rows are left stale;
-// materialize_kernel rebuilds them when something else needs them.
-template <int KT, bool BF16, bool WD, bool SPARSE>
-__global__ void __launch_bounds__(kHotThreads, 2)
-merge_step_implicit_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m,
-                           int64_t stride, BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags,
-                           StepParams p)
+// ---------------------------------------------------------------------------- one round in one kernel
+// The local step of all K workers followed by the merge, in one pass over the index range
+// (Algorithm 2's "update replica" for every worker, then Algorithm 3 and the re-clone).
+// Per index: w and D are read once; for every worker, in the order i = 0..K-1, its gradient
+// and momentum are read, the step is taken in registers, the new momentum is stored and the
+// replica change r_i - w is added to the running sum; then Dnew = sum / K, w and D are
+// written.  The stepped replicas are never stored, because the merge re-clones them: after
+// the kernel every replica is w (a lazy clone, see merge_lazy_kernel).
+//   FROM_W: every replica is still the clone of w when the round starts (exactly one local
+//           step per worker and period, the usual case): the step starts from w in registers
+//           and no replica row is read.  Per index the kernel then moves
+//           16 + K * (g + 8) bytes with momentum (16 + K * g for plain SGD): w, D, K m, K g in;
+//           w, D, K m out.  Otherwise replica i is read from gp.r_src[i] (its row, or w).
+// Same operations in the same order as local_step_kernel for every worker followed by
+// merge_kernel, so the results are bit-identical.  Workers are handled B at a time: all
+// loads of a batch are requested before the first use.
+template <int NB, bool FIRST, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+__device__ __forceinline__ void round_batch(f8& acc, const f8& wv, float* __restrict__ m, int64_t stride, int i0,
+                                            const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp,
+                                            int64_t o, const StepParams& p)
 {
-    static_assert(KT > 0, "the momentum rows of all workers are held in registers");
-    constexpr int B = KT < 8 ? KT : 8;           // workers whose gradients are in flight together
-    const float fK = (float)KT;
+    const int64_t e = o * 8;
+    int32_t sl[NB];
+    if (SPARSE && sp.inside) {
+#pragma unroll
+        for (int b = 0; b < NB; ++b) sl[b] = __ldg(gp.slot[i0 + b] + sp.row);
+    }
+    GradRaw<BF16> graw[NB];
+    f8 mm[NB];
+    f8 rr[FROM_W ? 1 : NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[b] : 0, i0 + b, o);
+        if (MOM) mm[b] = ld8(m + (int64_t)(i0 + b) * stride + e);
+        if (!FROM_W) rr[b] = ld8(gp.r_src[i0 + b] + e);
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        const f8 gg = widen_grad<BF16>(graw[b]);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float r_old = FROM_W ? wv.v[q] : rr[FROM_W ? 0 : b].v[q];
+            const float r_new = step1<MOM, WD>(gg.v[q], mm[b].v[q], r_old, p);
+            const float change = __fsub_rn(r_new, wv.v[q]);
+            acc.v[q] = (FIRST && b == 0) ? change : __fadd_rn(acc.v[q], change);
+        }
+        if (MOM) st8(m + (int64_t)(i0 + b) * stride + e, mm[b]);
+    }
+}
+
+constexpr int kRoundBatchF32 = 8;    // workers in flight together: 16 x 32-byte loads per thread (g and m)
+constexpr int kRoundBatchBf16 = 8;
+
+template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+__global__ void __launch_bounds__(kHotThreads, 2)
+round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m, int64_t stride, int K,
+             BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags, StepParams p, int64_t lim)
+{
+    const float fK = (float)K;
     const int64_t step = (int64_t)gridDim.x * kHotThreads;
     for (int64_t o = o0 + (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < o0 + n; o += step) {
+        HPSGD_GUARD_GROUP(o, lim, kIdRound);
         const int64_t e = o * 8;
         SegPos sp{false, 0, 0};
-        int32_t sl[KT];
-        if (SPARSE) {
-            sp = seg_pos(seg, o);
-            if (sp.inside) {
-#pragma unroll
-                for (int i = 0; i < KT; ++i) sl[i] = __ldg(gp.slot[i] + sp.row);
-            }
-        }
+        if (SPARSE) sp = seg_pos(seg, o);
         const f8 wv = ld8(w + e);
         f8 dv = zero8();
         if (flags & kMergeApplyPending) dv = ld8(D + e);
-        f8 mv[KT];
-#pragma unroll
-        for (int i = 0; i < KT; ++i) mv[i] = ld8(m + (int64_t)i * stride + e);
-        // the gradients do not depend on the merge: the first batch is requested before it
-        GradRaw<BF16> graw[B];
-#pragma unroll
-        for (int b = 0; b < B; ++b) graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[b] : 0, b, o);
-        // ---- merge over the recomputed replicas r_i = w - mu*m_i
+        // ---- local steps and the running sum of replica changes, worker 0 first
         f8 acc;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) acc.v[q] = __fsub_rn(__fmaf_rn(p.neg_mu, mv[0].v[q], wv.v[q]), wv.v[q]);
-#pragma unroll
-        for (int i = 1; i < KT; ++i)
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                acc.v[q] = __fadd_rn(acc.v[q], __fsub_rn(__fmaf_rn(p.neg_mu, mv[i].v[q], wv.v[q]), wv.v[q]));
+        int i = 0;
+        if (K >= B) {
+            round_batch<B, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p);
+            i = B;
+        } else {
+            round_batch<1, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p);
+            i = 1;
+        }
+        for (; i + B <= K; i += B)
+            round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p);
+        for (; i < K; ++i)
+            round_batch<1, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p);
+        // ---- merge
         f8 dnew, wn;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -681,44 +808,6 @@ merge_step_implicit_kernel(float* __restrict__ w, float* __restrict__ D, float* 
         }
         st8(w + e, wn);
         st8(D + e, dnew);
-        // ---- local step from the clone wn: only the momentum is stored
-#pragma unroll
-        for (int i0 = 0; i0 < KT; i0 += B) {
-            if (i0 > 0) {
-#pragma unroll
-                for (int b = 0; b < B; ++b)
-                    graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[i0 + b] : 0, i0 + b, o);
-            }
-#pragma unroll
-            for (int b = 0; b < B; ++b) {
-                const f8 gg = widen_grad<BF16>(graw[b]);
-                f8 mn;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float gd = WD ? __fmaf_rn(p.lambda, wn.v[q], gg.v[q]) : gg.v[q];
-                    mn.v[q] = __fmaf_rn(p.beta, mv[i0 + b].v[q], gd);
-                }
-                st8(m + (int64_t)(i0 + b) * stride + e, mn);
-            }
-        }
-    }
-}
-
-// r_i = fma(-mu, m_i, w) for every worker (blockIdx.y): rebuilds replica rows left stale by
-// merge_step_implicit_kernel.
-__global__ void __launch_bounds__(kHotThreads)
-materialize_kernel(const float* __restrict__ w, const float* __restrict__ m, float* __restrict__ r,
-                   int64_t stride, int64_t n, float neg_mu)
-{
-    const int64_t off = (int64_t)blockIdx.y * stride;
-    const int64_t step = (int64_t)gridDim.x * kHotThreads;
-    for (int64_t o = (int64_t)blockIdx.x * kHotThreads + threadIdx.x; o < n; o += step) {
-        const f8 wv = ld8(w + o * 8);
-        const f8 mv = ld8(m + off + o * 8);
-        f8 rr;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) rr.v[q] = __fmaf_rn(neg_mu, mv.v[q], wv.v[q]);
-        st8(r + off + o * 8, rr);
     }
 }
 

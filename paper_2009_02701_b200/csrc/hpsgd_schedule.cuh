@@ -14,21 +14,52 @@ int wait_pending_d2h(cudaStream_t s)
     return HPSGD_OK;
 }
 
-// Rebuild replica rows that the implicit-replica kernel left stale: r_i = fma(-mu, m_i, w).
-int ensure_replicas()
+// Lazy clones (HPSGD_OPT_FUSE = 2): a merge does not write the K re-cloned replicas; a replica
+// that nothing has stepped since is read from w.  Needs one pointer per worker in the launch.
+bool lazy_clones()
 {
-    if (!g.replicas_stale) return HPSGD_OK;
-    const int64_t n = g.P_pad / 8;
-    dim3 grid(hot_grid(n), g.K);
-    materialize_kernel<<<grid, kHotThreads, 0, g.main>>>(g.w, g.m, g.r, g.stride, n, -g.lr);
-    ++g.launches;
-    g.replicas_stale = false;
+    return g.fuse == 2 && g.form == HPSGD_FORM_REPLICA_CHANGE && !g.pipeline && g.K <= kMaxBatch;
+}
+
+// Where replica i is read from (not for the pipelined schedule, which keeps its own books).
+const float* replica_src(int i)
+{
+    return g.row_valid[i] ? g.r + (int64_t)i * g.stride : g.w;
+}
+
+// Write the rows of replicas that are lazy clones (r_i = w), for a schedule that reads rows.
+int materialize_clones()
+{
+    bool any = false;
+    for (int i = 0; i < g.K; ++i) any = any || !g.row_valid[i];
+    if (!any) return HPSGD_OK;
+    for (int c = 0; c < g.chunks; ++c)
+        if (g.merge_unwaited[c]) {             // w is last written by a merge on the side stream
+            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
+            g.merge_unwaited[c] = 0;
+        }
+    for (int i = 0; i < g.K; ++i) {
+        if (g.row_valid[i]) continue;
+        CUDA_TRY(cudaMemcpyAsync(g.r + (int64_t)i * g.stride, g.w, (size_t)g.P_pad * 4, cudaMemcpyDeviceToDevice, g.main));
+        g.row_valid[i] = 1;
+    }
     if (g.overlap)
         for (int c = 0; c < g.chunks; ++c) {
             CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
             g.local_recorded[c] = 1;
         }
-    return check_async();
+    return HPSGD_OK;
+}
+
+SparseSeg sparse_seg(bool sparse)
+{
+    SparseSeg seg{0, 0, 1};
+    if (sparse) {
+        seg.o_begin = g.offsets[g.sp_tensor] / 8;
+        seg.o_end = seg.o_begin + g.sp_rows * g.sp_cols / 8;
+        seg.cols8 = (int32_t)(g.sp_cols / 8);
+    }
+    return seg;
 }
 
 // ---------------------------------------------------------------------------- local step
@@ -45,7 +76,7 @@ void launch_local(const LocalLaunch& L)
 {
     dim3 grid(hot_grid(L.n), L.nw);
     local_step_kernel<BF16, MOM, WD, SPARSE><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp,
-                                                                               L.seg, L.o0, L.n, L.p);
+                                                                               L.seg, L.o0, L.n, L.p, group_limit());
 }
 
 template <bool BF16, bool MOM, bool WD>
@@ -69,8 +100,9 @@ void launch_accum_step(bool sparse, const LocalLaunch& L)
 {
     dim3 grid(hot_grid(L.n), L.nw);
     const bool bf = g.grad_dtype == HPSGD_BF16;
-#define HPSGD_ACCUM_CASE(B, S) \
-    accum_step_kernel<B, S><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.o0, L.n, L.p.neg_mu)
+#define HPSGD_ACCUM_CASE(B, S)                                                                                  \
+    accum_step_kernel<B, S><<<grid, kHotThreads, 0, g.main>>>(g.r, g.m, g.stride, L.w0, L.gp, L.seg, L.o0, L.n, \
+                                                              L.p.neg_mu, group_limit())
     if (bf && sparse) HPSGD_ACCUM_CASE(true, true);
     else if (bf) HPSGD_ACCUM_CASE(true, false);
     else if (sparse) HPSGD_ACCUM_CASE(false, true);
@@ -81,8 +113,6 @@ void launch_accum_step(bool sparse, const LocalLaunch& L)
 // Enqueue the local step of workers [w0, w0 + nw) on the main stream, chunk by chunk.
 int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
 {
-    TRY(ensure_replicas());
-    for (int i = 0; i < nw; ++i) g.steps_in_period[w0 + i] += 1;
     LocalLaunch L{};
     L.w0 = w0; L.nw = nw; L.gp = gp;
     if (g.pipeline) {
@@ -93,14 +123,15 @@ int enqueue_local(int w0, int nw, const BatchPtrs& gp, bool sparse)
                 g.touched[w0 + i] = 1;
             }
         }
+    } else {
+        for (int i = 0; i < nw; ++i) {
+            if (!g.row_valid[w0 + i]) L.gp.r_src[i] = g.w;      // a lazy clone: the step writes its row
+            g.row_valid[w0 + i] = 1;
+            g.at_w[w0 + i] = 0;
+        }
     }
     L.p = StepParams{-g.lr, g.beta, g.lambda};
-    L.seg = SparseSeg{0, 0, 1};
-    if (sparse) {
-        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
-        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
-        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
-    }
+    L.seg = sparse_seg(sparse);
     const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
     for (int c = 0; c < g.chunks; ++c) {
         int64_t lo, hi;
@@ -142,6 +173,7 @@ int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* g
         sb.n_rows[i] = (d.row_idx && d.n_rows > 0) ? d.n_rows : 0;
         most = std::max(most, sb.n_rows[i]);
         gp->slot[i] = sb.slot[i];
+        gp->n_rows[i] = sb.n_rows[i];
         gp->row_vals[i] = d.row_vals;
         gp->dense[i] = d.dense;
     }
@@ -152,24 +184,35 @@ int enqueue_slot_maps(int w0, int nw, const hpsgd_grad_desc* descs, BatchPtrs* g
     return HPSGD_OK;
 }
 
+// ---------------------------------------------------------------------------- merge
 template <int KT>
 void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
 {
-    merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags);
+    merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags, group_limit());
+}
+
+template <int KT>
+void launch_merge_lazy(cudaStream_t s, const ReducePtrs& rp, int64_t o0, int64_t n, int flags)
+{
+    merge_lazy_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, rp, g.K, o0, n, flags, group_limit());
 }
 
 template <int KT>
 void launch_accum_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
 {
-    accum_merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.m, g.stride, g.K, o0, n, flags, -g.lr);
+    accum_merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.m, g.stride, g.K, o0, n, flags, -g.lr,
+                                                               group_limit());
 }
 
 // Enqueue one merge, chunk by chunk, on the side stream (main stream without overlap).
 int enqueue_merge(int flags)
 {
-    TRY(ensure_replicas());
     cudaStream_t s = g.overlap ? g.side : g.main;
     TRY(wait_pending_d2h(s));
+    const bool lazy = lazy_clones();
+    ReducePtrs rp{};
+    if (lazy)
+        for (int i = 0; i < g.K; ++i) rp.src[i] = replica_src(i);
     for (int c = 0; c < g.chunks; ++c) {
         int64_t lo, hi;
         chunk_range(c, &lo, &hi);
@@ -187,6 +230,13 @@ int enqueue_merge(int flags)
             case 16: launch_accum_merge<16>(s, lo, hi - lo, flags); break;
             default: launch_accum_merge<0>(s, lo, hi - lo, flags); break;
             }
+        } else if (lazy) {
+            switch (g.K) {
+            case 4: launch_merge_lazy<4>(s, rp, lo, hi - lo, flags); break;
+            case 8: launch_merge_lazy<8>(s, rp, lo, hi - lo, flags); break;
+            case 16: launch_merge_lazy<16>(s, rp, lo, hi - lo, flags); break;
+            default: launch_merge_lazy<0>(s, rp, lo, hi - lo, flags); break;
+            }
         } else {
             switch (g.K) {
             case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
@@ -202,13 +252,15 @@ int enqueue_merge(int flags)
             g.merge_unwaited[c] = 1;
         }
     }
+    std::fill(g.at_w.begin(), g.at_w.end(), 1);
+    std::fill(g.row_valid.begin(), g.row_valid.end(), lazy ? 0 : 1);
     return check_async();
 }
 
 template <int KT>
 void launch_reduce(const float* w_old, const ReducePtrs& rp, int64_t n)
 {
-    reduce_kernel<KT><<<hot_grid(n), kHotThreads, 0, g.side>>>(w_old, g.D, rp, g.K, n);
+    reduce_kernel<KT><<<hot_grid(n), kHotThreads, 0, g.side>>>(w_old, g.D, rp, g.K, n, group_limit());
 }
 
 // Pipelined synchronisation: the commit w_next = w + D runs on the main stream, in order with
@@ -226,7 +278,7 @@ int enqueue_pipelined_merge(int flags)
     }
     EventPair ep{};
     TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE, &ep));
-    commit_kernel<<<hot_grid(n), kHotThreads, 0, g.main>>>(g.wbuf[g.cur], g.D, g.wbuf[nxt], n, flags);
+    commit_kernel<<<hot_grid(n), kHotThreads, 0, g.main>>>(g.wbuf[g.cur], g.D, g.wbuf[nxt], n, flags, group_limit());
     ++g.launches;
     TRY(prof_end(g.main, &ep));
     CUDA_TRY(cudaEventRecord(g.ev_commit, g.main));
@@ -253,12 +305,19 @@ int enqueue_pipelined_merge(int flags)
     return check_async();
 }
 
-// A merge that hpsgd_sync_merge deferred (fuse option) and that nothing has absorbed yet.
+// Work that an earlier call held back (HPSGD_OPT_FUSE) and that nothing has absorbed: a merge
+// (fuse 1) runs on its own, a batched local step (fuse 2) runs as an ordinary local step.
 int flush_deferred()
 {
-    if (!g.merge_deferred) return HPSGD_OK;
-    g.merge_deferred = false;
-    return enqueue_merge(g.deferred_flags);
+    if (g.merge_deferred) {
+        g.merge_deferred = false;
+        TRY(enqueue_merge(g.deferred_flags));
+    }
+    if (g.step_deferred) {
+        g.step_deferred = false;
+        TRY(enqueue_local(0, g.K, g.deferred_gp, g.deferred_sparse));
+    }
+    return HPSGD_OK;
 }
 
 struct FusedLaunch {
@@ -269,11 +328,12 @@ struct FusedLaunch {
     StepParams p;
 };
 
+// ---------------------------------------------------------------------------- fuse 1: merge + next local step
 template <int KT, bool BF16, bool MOM, bool WD, bool SPARSE>
 void launch_fused(const FusedLaunch& L)
 {
     merge_step_kernel<KT, BF16, MOM, WD, SPARSE><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
-        g.w, g.D, g.r, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p);
+        g.w, g.D, g.r, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
 }
 
 template <int KT, bool BF16>
@@ -302,46 +362,15 @@ void launch_fused_k(bool mom, bool wd, bool sparse, const FusedLaunch& L)
     }
 }
 
-template <int KT>
-void launch_implicit(bool sparse, const FusedLaunch& L)
-{
-    const bool bf = g.grad_dtype == HPSGD_BF16, wd = g.lambda != 0.f;
-#define HPSGD_IMPLICIT_CASE(B, W, S)                                                                     \
-    merge_step_implicit_kernel<KT, B, W, S><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(                \
-        g.w, g.D, g.m, g.stride, L.gp, L.seg, L.o0, L.n, L.flags, L.p)
-    if (bf) {
-        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(true, true, true); else HPSGD_IMPLICIT_CASE(true, true, false); }
-        else { if (sparse) HPSGD_IMPLICIT_CASE(true, false, true); else HPSGD_IMPLICIT_CASE(true, false, false); }
-    } else {
-        if (wd) { if (sparse) HPSGD_IMPLICIT_CASE(false, true, true); else HPSGD_IMPLICIT_CASE(false, true, false); }
-        else { if (sparse) HPSGD_IMPLICIT_CASE(false, false, true); else HPSGD_IMPLICIT_CASE(false, false, false); }
-    }
-#undef HPSGD_IMPLICIT_CASE
-}
-
-// Can the deferred merge and the coming batched step run with the replicas left implicit?
-bool implicit_ok()
-{
-    return g.fuse == 2 && g.deferred_all_single && g.beta != 0.f && (g.K == 4 || g.K == 8 || g.K == 16);
-}
-
 // The deferred merge and the local step of all K workers in one kernel per chunk (main stream).
 int enqueue_fused(const BatchPtrs& gp, bool sparse)
 {
-    const bool implicit = implicit_ok();
-    if (!implicit) TRY(ensure_replicas());
     TRY(wait_pending_d2h(g.main));
-    for (int i = 0; i < g.K; ++i) g.steps_in_period[i] += 1;
     FusedLaunch L{};
     L.gp = gp;
     L.flags = g.deferred_flags;
     L.p = StepParams{-g.lr, g.beta, g.lambda};
-    L.seg = SparseSeg{0, 0, 1};
-    if (sparse) {
-        L.seg.o_begin = g.offsets[g.sp_tensor] / 8;
-        L.seg.o_end = L.seg.o_begin + g.sp_rows * g.sp_cols / 8;
-        L.seg.cols8 = (int32_t)(g.sp_cols / 8);
-    }
+    L.seg = sparse_seg(sparse);
     g.merge_deferred = false;
     const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
     for (int c = 0; c < g.chunks; ++c) {
@@ -355,13 +384,7 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
         L.o0 = lo; L.n = hi - lo;
         EventPair ep{};
         TRY(prof_begin(g.main, HPSGD_KERNEL_MERGE_STEP, &ep));
-        if (implicit) {
-            switch (g.K) {
-            case 4: launch_implicit<4>(sparse, L); break;
-            case 8: launch_implicit<8>(sparse, L); break;
-            default: launch_implicit<16>(sparse, L); break;
-            }
-        } else if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
+        if (g.grad_dtype == HPSGD_BF16) launch_fused_k<true>(mom, wd, sparse, L);
         else launch_fused_k<false>(mom, wd, sparse, L);
         ++g.launches;
         TRY(prof_end(g.main, &ep));
@@ -370,7 +393,81 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
             g.local_recorded[c] = 1;
         }
     }
-    g.replicas_stale = implicit;
+    std::fill(g.at_w.begin(), g.at_w.end(), 0);          // merged, re-cloned and stepped once
+    return check_async();
+}
+
+// ---------------------------------------------------------------------------- fuse 2: local step + merge, one round
+// Workers whose loads are in flight together: 8 (fp32 gradients, 16 x 32 bytes per thread) or
+// 16 with bf16 gradients (half the gradient bytes).
+template <bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+void launch_round(const FusedLaunch& L)
+{
+    constexpr int B = BF16 ? kRoundBatchBf16 : kRoundBatchF32;
+    round_kernel<B, BF16, MOM, WD, SPARSE, FROM_W><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
+        g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
+}
+
+template <bool BF16, bool MOM, bool WD>
+void launch_round_s(bool sparse, bool from_w, const FusedLaunch& L)
+{
+    if (sparse) {
+        if (from_w) launch_round<BF16, MOM, WD, true, true>(L);
+        else launch_round<BF16, MOM, WD, true, false>(L);
+    } else {
+        if (from_w) launch_round<BF16, MOM, WD, false, true>(L);
+        else launch_round<BF16, MOM, WD, false, false>(L);
+    }
+}
+
+template <bool BF16>
+void launch_round_d(bool mom, bool wd, bool sparse, bool from_w, const FusedLaunch& L)
+{
+    if (mom && wd) launch_round_s<BF16, true, true>(sparse, from_w, L);
+    else if (mom) launch_round_s<BF16, true, false>(sparse, from_w, L);
+    else if (wd) launch_round_s<BF16, false, true>(sparse, from_w, L);
+    else launch_round_s<BF16, false, false>(sparse, from_w, L);
+}
+
+// The deferred batched local step and the merge that follows it in one kernel per chunk (main
+// stream).  Afterwards every replica is a lazy clone of the new w.
+int enqueue_round(int flags)
+{
+    TRY(wait_pending_d2h(g.main));
+    g.step_deferred = false;
+    FusedLaunch L{};
+    L.gp = g.deferred_gp;
+    bool from_w = true;
+    for (int i = 0; i < g.K; ++i) {
+        from_w = from_w && g.at_w[i];
+        L.gp.r_src[i] = replica_src(i);
+    }
+    L.flags = flags;
+    L.p = StepParams{-g.lr, g.beta, g.lambda};
+    L.seg = sparse_seg(g.deferred_sparse);
+    const bool mom = g.beta != 0.f, wd = g.lambda != 0.f;
+    for (int c = 0; c < g.chunks; ++c) {
+        int64_t lo, hi;
+        chunk_range(c, &lo, &hi);
+        if (hi <= lo) continue;
+        if (g.merge_unwaited[c]) {
+            CUDA_TRY(cudaStreamWaitEvent(g.main, g.ev_merge[c], 0));
+            g.merge_unwaited[c] = 0;
+        }
+        L.o0 = lo; L.n = hi - lo;
+        EventPair ep{};
+        TRY(prof_begin(g.main, HPSGD_KERNEL_ROUND, &ep));
+        if (g.grad_dtype == HPSGD_BF16) launch_round_d<true>(mom, wd, g.deferred_sparse, from_w, L);
+        else launch_round_d<false>(mom, wd, g.deferred_sparse, from_w, L);
+        ++g.launches;
+        TRY(prof_end(g.main, &ep));
+        if (g.overlap) {
+            CUDA_TRY(cudaEventRecord(g.ev_local[c], g.main));
+            g.local_recorded[c] = 1;
+        }
+    }
+    std::fill(g.at_w.begin(), g.at_w.end(), 1);
+    std::fill(g.row_valid.begin(), g.row_valid.end(), 0);
     return check_async();
 }
 

@@ -9,6 +9,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "hpsgd_kernels.cuh"
@@ -39,11 +40,15 @@ int fail(int code, const char* fmt, ...)
     return code;
 }
 
+// A failed call is reported once: cudaGetLastError also clears a non-sticky error, so that the
+// next, valid call is not blamed for it.
 #define CUDA_TRY(expr)                                                                      \
     do {                                                                                    \
         cudaError_t e_ = (expr);                                                            \
-        if (e_ != cudaSuccess)                                                              \
+        if (e_ != cudaSuccess) {                                                            \
+            cudaGetLastError();                                                             \
             return fail(HPSGD_E_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));      \
+        }                                                                                   \
     } while (0)
 
 #define TRY(expr)                \
@@ -102,11 +107,13 @@ struct Ctx {
     std::vector<char> touched;             // pipeline: worker has made a local step this period
     cudaEvent_t ev_commit = nullptr, ev_reduce = nullptr;
     bool reduce_outstanding = false;
-    bool merge_deferred = false;           // hpsgd_sync_merge was called but its merge not yet enqueued
+    bool merge_deferred = false;           // fuse 1: hpsgd_sync_merge was called but its merge not yet enqueued
     int deferred_flags = 0;
-    std::vector<int> steps_in_period;      // local steps of each worker since the last merge request
-    bool deferred_all_single = false;      // every worker made exactly one step in the period the deferred merge closes
-    bool replicas_stale = false;           // replica rows not written by the implicit-replica kernel
+    bool step_deferred = false;            // fuse 2: a batched local step waits for the merge it will run with
+    BatchPtrs deferred_gp{};               //         its gradient pointers
+    bool deferred_sparse = false;
+    std::vector<char> at_w;                // replica i equals w: no local step since its last clone
+    std::vector<char> row_valid;           // row i of r holds replica i (else it is a lazy clone: read w)
     int64_t launches = 0;
     int sm_count = 148;
     int sp_tensor = -1;                    // sparse-row tensor
@@ -116,14 +123,36 @@ struct Ctx {
     bool stage_used[2] = {false, false};
     int stage_next = 0;
     std::vector<EventPair> prof;           // profiling
-    double prof_ms[3] = {0, 0, 0};
-    int64_t prof_launches[3] = {0, 0, 0};
+    double prof_ms[4] = {0, 0, 0, 0};
+    int64_t prof_launches[4] = {0, 0, 0, 0};
+    int64_t debug_limit = -1;              // checked build: groups per flat buffer the kernels test against (< 0: P_pad / 8)
 } g;
 
 int check_async()
 {
-    cudaError_t e = cudaPeekAtLastError();
+    cudaError_t e = cudaGetLastError();     // reported once, then cleared (a sticky error comes back by itself)
     if (e != cudaSuccess) return fail(HPSGD_E_CUDA, "CUDA error: %s", cudaGetErrorString(e));
+    return HPSGD_OK;
+}
+
+// Groups of 8 elements in a flat buffer: what the guards of the checked build test against.
+int64_t group_limit() { return g.debug_limit >= 0 ? g.debug_limit : g.P_pad / 8; }
+
+// Checked build: fetch and clear the record a kernel guard left behind.  Called where the host
+// has just waited for the device, so the copy costs nothing extra.
+int debug_poll()
+{
+#ifdef HPSGD_DEBUG
+    DebugReport rep{};
+    CUDA_TRY(cudaMemcpyFromSymbol(&rep, g_debug_report, sizeof rep));
+    if (rep.code != 0) {
+        const DebugReport zero{};
+        CUDA_TRY(cudaMemcpyToSymbol(g_debug_report, &zero, sizeof zero));
+        static const char* what[] = {"", "group index", "row -> slot entry", "row index"};
+        return fail(HPSGD_E_CUDA, "checked build: kernel %d met %s %lld outside [0, %lld); the access was skipped",
+                    rep.kernel, what[rep.code < 4 ? rep.code : 0], rep.index, rep.limit);
+    }
+#endif
     return HPSGD_OK;
 }
 
@@ -241,6 +270,31 @@ int check_desc(const hpsgd_grad_desc* d)
     return HPSGD_OK;
 }
 
+// Checked build: the listed rows of a sparse-row gradient are copied to the host and tested
+// (ascending, hence unique, and inside [0, rows)) before anything is enqueued for them.  The
+// copy is ordered behind the work already on `s`, which may still be producing the list.  The
+// normal build trusts the caller, as the contract says, and does nothing here.
+int validate_rows(const hpsgd_grad_desc* d, int64_t rows, cudaStream_t s)
+{
+#ifdef HPSGD_DEBUG
+    if (!d->row_idx || d->n_rows <= 0) return HPSGD_OK;
+    std::vector<int32_t> idx((size_t)d->n_rows);
+    CUDA_TRY(cudaMemcpyAsync(idx.data(), d->row_idx, idx.size() * 4, cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    for (size_t k = 0; k < idx.size(); ++k) {
+        if (idx[k] < 0 || idx[k] >= rows)
+            return fail(HPSGD_E_BADARG, "row_idx[%zu] = %d is outside [0, %lld)", k, idx[k], (long long)rows);
+        if (k > 0 && idx[k] == idx[k - 1])
+            return fail(HPSGD_E_BADARG, "row_idx[%zu] = %d is listed twice", k, idx[k]);
+        if (k > 0 && idx[k] < idx[k - 1])
+            return fail(HPSGD_E_BADARG, "row_idx is not ascending at entry %zu (%d after %d)", k, idx[k], idx[k - 1]);
+    }
+#else
+    (void)d; (void)rows; (void)s;
+#endif
+    return HPSGD_OK;
+}
+
 int need_init()
 {
     if (!g.inited) return fail(HPSGD_E_STATE, "hpsgd_init has not been called");
@@ -260,7 +314,7 @@ int sync_all()
     if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
     if (g.d2h) CUDA_TRY(cudaStreamSynchronize(g.d2h));
     g.d2h_outstanding = false;
-    return HPSGD_OK;
+    return debug_poll();
 }
 
 int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; blocking
@@ -275,13 +329,13 @@ int reset_state_from_w()     // D = 0, r_i = w, m_i = 0, counters cleared; block
         const int64_t nvec = g.P_pad / 4;
         clone_kernel<<<grid_for(clone_kernel, nvec, kThreads), kThreads, 0, g.main>>>(g.w, g.r, g.stride, g.K, nvec);
         ++g.launches;
-        CUDA_TRY(cudaGetLastError());
+        TRY(check_async());
     }
     CUDA_TRY(cudaStreamSynchronize(g.main));
     g.D_valid = false;
     g.merges = 0;
-    g.replicas_stale = false;
-    std::fill(g.steps_in_period.begin(), g.steps_in_period.end(), 0);
+    std::fill(g.at_w.begin(), g.at_w.end(), 1);
+    std::fill(g.row_valid.begin(), g.row_valid.end(), 1);
     std::fill(g.local_recorded.begin(), g.local_recorded.end(), 0);
     std::fill(g.merge_unwaited.begin(), g.merge_unwaited.end(), 0);
     return HPSGD_OK;

@@ -27,6 +27,11 @@ def dev_view(addr: int, n: int, typestr="<f4") -> torch.Tensor:
     return torch.as_tensor(_RawDeviceArray(addr, n, typestr), device=DEV).clone()
 
 
+def dev_tensor(addr: int, n: int, typestr="<f4") -> torch.Tensor:
+    """The n elements at a raw device address as a torch tensor that aliases them (no copy)."""
+    return torch.as_tensor(_RawDeviceArray(addr, n, typestr), device=DEV)
+
+
 def to_device(a: np.ndarray) -> torch.Tensor:
     """Upload a numpy array (fp32, or uint16 bf16 bit patterns, or int32)."""
     if a.dtype == np.uint16:

@@ -384,11 +384,11 @@ def test_pipelined_sync_argument_checks():
 
 
 # ---------------------------------------------------------------- checkpoint
-@pytest.mark.parametrize("mode", ["plain", "fuse", "implicit", "pipeline", "accum"])
+@pytest.mark.parametrize("mode", ["plain", "fuse", "round", "pipeline", "accum"])
 def test_export_import_resumes_bit_identically(mode):
     momentum = 0.0 if mode == "accum" else 0.9
     cfg = small("ckpt", 4, [20_000, 77], T=6, momentum=momentum, lr=0.05)
-    kw = dict(fuse={"fuse": 1, "implicit": 2}.get(mode, 0), pipeline=int(mode == "pipeline"),
+    kw = dict(fuse={"fuse": 1, "round": 2}.get(mode, 0), pipeline=int(mode == "pipeline"),
               form=hp.HPSGD_FORM_GRADIENT_ACCUMULATION if mode == "accum" else 0)
 
     def rounds(t0, t1, keep):
@@ -426,52 +426,112 @@ def test_more_workers_than_one_batched_launch_addresses():
     cfg = small("k40", 40, [5000, 33], T=3, momentum=0.9)
     gu.run_both(cfg, cfg.T, batched=True)
     gu.run_both(cfg, cfg.T, batched=True, fuse=1, chunks=2)
+    gu.run_both(cfg, cfg.T, batched=True, fuse=2)
     gu.run_both(cfg, cfg.T, batched=False)
 
 
-# ---------------------------------------------------------------- fused merge + step with implicit replicas
+# ---------------------------------------------------------------- one kernel per round, lazy clones
 @pytest.mark.parametrize("K,momentum,wd,staleness,H", [(16, 0.9, 0.0, 1, 1), (8, 0.9, 5e-4, 1, 1), (4, 0.5, 1e-3, 0, 1),
-                                                        (16, 0.9, 0.0, 1, 2), (3, 0.9, 0.0, 1, 1), (8, 0.0, 0.0, 1, 1)])
-def test_implicit_replicas_match_oracle(K, momentum, wd, staleness, H):
-    """HPSGD_OPT_FUSE = 2: replicas recomputed as fma(-mu, m, w) where that is exact; K = 3, plain SGD
-    and several steps per period take the ordinary fused path; all of it bit-identical."""
-    cfg = small("implicit", K, [70_001, 33, 4096], T=6, momentum=momentum, wd=wd, staleness=staleness)
+                                                        (16, 0.9, 0.0, 1, 2), (3, 0.9, 0.0, 1, 1), (8, 0.0, 0.0, 1, 1),
+                                                        (1, 0.9, 0.0, 1, 1), (5, 0.0, 1e-3, 0, 3), (9, 0.9, 0.0, 1, 1),
+                                                        (32, 0.9, 0.0, 1, 1), (17, 0.0, 0.0, 1, 2)])
+def test_round_kernel_matches_oracle(K, momentum, wd, staleness, H):
+    """HPSGD_OPT_FUSE = 2: the batched local step runs inside the kernel of the merge that follows it
+    and no replica row is written; with several steps per period only the last one is fused and the
+    earlier ones read w (the lazy clone) or their row.  All of it bit-identical."""
+    cfg = small("round", K, [70_001, 33, 4096], T=6, momentum=momentum, wd=wd, staleness=staleness)
     gu.run_both(cfg, cfg.T, staleness=staleness, fuse=2, batched=True, chunks=2, steps_per_round=H)
+    gu.run_both(cfg, 3, staleness=staleness, fuse=2, batched=True, steps_per_round=H, check_each_round=True,
+                session_kw=dict(lend_arena=True, canary=True, streams=True))
+
+
+@pytest.mark.parametrize("P", [1, 31, 33, 129, 1000, 4097])
+def test_round_kernel_odd_sizes(P):
+    for K, momentum in ((2, 0.9), (7, 0.0), (16, 0.9)):
+        cfg = small("round_odd", K, [P], T=3, momentum=momentum)
+        gu.run_both(cfg, cfg.T, fuse=2, batched=True, check_each_round=True)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_implicit_replicas_sparse_rows(dtype):
-    cfg = small("implicit_sparse", 4, [1000, 300 * 64, 777, 64], T=5, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
-    gu.run_both(cfg, cfg.T, fuse=2, batched=True)
+@pytest.mark.parametrize("batched", [True, False])
+def test_round_kernel_sparse_rows(dtype, batched):
+    cfg = small("round_sparse", 4, [1000, 300 * 64, 777, 64], T=5, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
+    gu.run_both(cfg, cfg.T, fuse=2, batched=batched)
+    cfg = small("round_sparse16", 16, [64, 200 * 128, 5], T=4, dtype=dtype, sparse=(1, 200, 128), scale=1e-3, wd=1e-4)
+    gu.run_both(cfg, cfg.T, fuse=2, batched=batched, chunks=3)
 
 
-def test_implicit_replicas_are_rebuilt_on_demand():
-    """Interleave implicit rounds with calls that need real replica rows."""
-    cfg = small("implicit_mixed", 8, [40_000, 17], T=8, momentum=0.9, wd=1e-4)
+def test_round_kernel_launches_one_kernel_per_round_and_writes_no_replica_row():
+    cfg = small("round_count", 8, [50_000], T=4)
+    with gu.session(cfg, fuse=2, lend_arena=True):
+        stacked = np.stack([gu.host_inputs(cfg, i, 0)["padded"] for i in range(cfg.K)])
+        g = gu.to_device(stacked.reshape(-1))
+        rows = []
+        for i in range(cfg.K):
+            r, _ = hp.hpsgd_get_replica(i)               # before any merge the rows are real
+            rows.append(r)
+        assert len(set(rows)) == cfg.K and hp.hpsgd_get_global() not in rows
+        poison = torch.full((cfg.layout.P_pad,), float("nan"), dtype=torch.float32, device=gu.DEV)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)
+        base = hp.hpsgd_launch_count()
+        for t in range(4):
+            hp.hpsgd_local_step_all(g, stacked.shape[1] * 4)
+            assert hp.hpsgd_launch_count() - base == t          # held back
+            hp.hpsgd_sync_merge()
+            assert hp.hpsgd_launch_count() - base == t + 1      # one kernel: K local steps + the merge
+            if t == 0:
+                # from here on the rows are dead storage: whatever they hold must never be read
+                hp.hpsgd_synchronize()
+                for r in rows:
+                    gu.dev_tensor(r, cfg.layout.P_pad).copy_(poison)
+                torch.cuda.synchronize()
+        hp.hpsgd_flush()
+        assert hp.hpsgd_launch_count() - base == 4
+        assert hp.hpsgd_profile_read(hp.HPSGD_KERNEL_ROUND)[1] == 4
+        assert hp.hpsgd_profile_read(hp.HPSGD_KERNEL_LOCAL_STEP)[1] == 0
+        assert hp.hpsgd_profile_read(hp.HPSGD_KERNEL_MERGE)[1] == 0
+        w = hp.hpsgd_get_global()
+        for i in range(cfg.K):
+            assert hp.hpsgd_get_replica(i)[0] == w               # lazy clones: the replica is w itself
+        for r in rows:
+            assert bool(torch.isnan(gu.dev_tensor(r, cfg.layout.P_pad)).all()), "a replica row was written"
+        assert bool(torch.isfinite(gu.dev_tensor(w, cfg.layout.P_pad)).all())
+
+
+def test_lazy_clones_under_every_other_call():
+    """Interleave whole-round kernels with per-worker steps, idle workers, merges on their own,
+    inspection and a change of schedule: replicas that exist only as 'w' must behave like rows."""
+    cfg = small("round_mixed", 8, [40_000, 17], T=10, momentum=0.9, wd=1e-4)
     o = gu.oracle_for(cfg)
-    with gu.session(cfg, fuse=2):
+    with gu.session(cfg, fuse=2, chunks=2):
         keep = []
-        launches = []
         for t in range(cfg.T):
             inputs = [gu.host_inputs(cfg, i, t) for i in range(cfg.K)]
-            for i, inp in enumerate(inputs):
-                o.local_step(i, inp["flat"])
-            if t == 4:                                   # per-worker calls in the middle of implicit rounds
+            if t in (4, 7):                              # per-worker calls; in round 7 worker 3 sits out
                 for i, inp in enumerate(inputs):
+                    if t == 7 and i == 3:
+                        continue
                     gu.gpu_step(cfg, i, inp, keep)
+                    o.local_step(i, inp["flat"])
             else:
                 stacked = np.stack([inp["padded"] for inp in inputs])
                 keep.append(gu.to_device(stacked.reshape(-1)))
-                before = hp.hpsgd_launch_count()
                 hp.hpsgd_local_step_all(keep[-1], stacked.shape[1] * 4)
-                launches.append(hp.hpsgd_launch_count() - before)
+                for i, inp in enumerate(inputs):
+                    o.local_step(i, inp["flat"])
             if t == 2:                                   # look at the replicas between step and merge
                 w, D, rs, ms = gu.gpu_state(cfg)
                 for i in range(cfg.K):
-                    gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d rebuilt from momentum" % i)
+                    gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d after a flushed step" % i)
+            if t == 5:
+                hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, 1)    # rows are written out, the other fused schedule takes over
+            if t == 8:
+                hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, 2)
             hp.hpsgd_sync_merge()
             o.sync_merge()
-        assert launches[1] == 1 and launches[2] == 1     # one kernel per round while implicit
+            if t == 3:
+                hp.hpsgd_sync_merge()                    # a merge with no step before it
+                o.sync_merge()
         w, D, rs, ms = gu.gpu_state(cfg)
         gu.assert_bitwise(w, o.get_global(), "global model")
         gu.assert_bitwise(D, o.get_pending(), "pending change")
@@ -480,12 +540,55 @@ def test_implicit_replicas_are_rebuilt_on_demand():
             gu.assert_bitwise(ms[i], o.get_momentum(i), "momentum %d" % i)
 
 
-@pytest.mark.parametrize("mode", ["two_streams", "one_stream", "fuse", "pipeline"])
+def test_fill_global_reseeds_like_a_fresh_init():
+    """hpsgd_fill_global(seed): w from hash stream 2 of that seed, everything else as after hpsgd_init."""
+    cfg = small("fill", 4, [5000, 77, 33], T=2, momentum=0.9)
+    other = small("fill", 4, [5000, 77, 33], T=2, momentum=0.9, seed=cfg.seed + 1000)
+    with gu.session(other):
+        fresh = gu.gpu_state(other)
+    for fuse in (0, 2):
+        with gu.session(cfg, fuse=fuse):
+            keep = []
+            for t in range(2):                               # leave every buffer dirty
+                for i in range(cfg.K):
+                    gu.gpu_step(cfg, i, gu.host_inputs(cfg, i, t), keep)
+                hp.hpsgd_sync_merge()
+            hp.hpsgd_fill_global(other.seed)
+            assert hp.hpsgd_get_sizes()[3] == 0
+            w, D, rs, ms = gu.gpu_state(cfg)
+            gu.assert_bitwise(w, other.initial_global(), "re-seeded global model vs the host generator")
+            gu.assert_bitwise(w, fresh[0], "re-seeded global model vs a fresh hpsgd_init")
+            assert not D.any()
+            for i in range(cfg.K):
+                gu.assert_bitwise(rs[i], w, "replica %d after the re-seed" % i)
+                assert not ms[i].any()
+            # and the run that follows is the run of a fresh state with that seed
+            o = gu.oracle_for(other)
+            for t in range(3):
+                for i in range(cfg.K):
+                    inp = gu.host_inputs(other, i, t)
+                    gu.gpu_step(other, i, inp, keep)
+                    o.local_step(i, inp["flat"])
+                hp.hpsgd_sync_merge()
+                o.sync_merge()
+            gu.assert_bitwise(gu.gpu_state(cfg)[0], o.get_global(), "global model of the run after the re-seed")
+            # the device generator follows the new seed too
+            out = torch.empty(cfg.layout.P_pad, dtype=torch.float32, device=gu.DEV)
+            hp.hpsgd_gen_grads(out, 1, 3, hp.HPSGD_GEN_UNIFORM, 1e-2)
+            hp.hpsgd_synchronize()
+            import workloads.hashgen as hg
+            gu.assert_bitwise(cfg.layout.unpack(out.cpu().numpy()),
+                              hg.grad_uniform(other.seed, 3, 1, scale=1e-2, idx0=0, n=cfg.P), "gradients of the new seed")
+            o.close()
+
+
+@pytest.mark.parametrize("mode", ["two_streams", "one_stream", "fuse", "round", "pipeline"])
 def test_async_host_copy_sees_the_model_of_its_merge(mode):
     """hpsgd_copy_global_async after merge t must deliver w as of merge t, although later local
     steps and merges are enqueued before anything is waited for."""
     cfg = small("d2h", 4, [60_000, 99], T=5, momentum=0.9)
-    kw = dict(overlap=0 if mode == "one_stream" else 1, fuse=int(mode == "fuse"), pipeline=int(mode == "pipeline"))
+    kw = dict(overlap=0 if mode == "one_stream" else 1, fuse={"fuse": 1, "round": 2}.get(mode, 0),
+              pipeline=int(mode == "pipeline"))
     o = gu.oracle_for(cfg)
     outs = [torch.empty(cfg.P, dtype=torch.float32).pin_memory() for _ in range(cfg.T)]
     want = []
