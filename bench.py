@@ -282,6 +282,264 @@ def aggregate(dist, device, elapsed_ms, units):
 
 
 # ------------------------------------------------------------------------------ GPU arm
+class _RawDeviceArray:
+    """A raw device address as something torch.as_tensor can wrap (CUDA array interface)."""
+
+    def __init__(self, addr, n, typestr="<f4"):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(addr), False), "version": 2}
+
+
+def parity_sample(cfg, n_random=1 << 14, edge=32, seed=2024):
+    """Un-padded parameter indices the oracle recomputes: both ends of every tensor plus random ones."""
+    picks = []
+    for size, start in zip(cfg.layout.sizes, cfg.layout.starts):
+        e = min(edge, size)
+        picks += [np.arange(start, start + e), np.arange(start + size - e, start + size)]
+    picks.append(np.random.default_rng(seed).integers(0, cfg.P, size=n_random))
+    return np.unique(np.concatenate(picks)).astype(np.int64)
+
+
+def ulp_distance(a, b):
+    a = np.ascontiguousarray(a, dtype=np.float32).view(np.int32).astype(np.int64)
+    b = np.ascontiguousarray(b, dtype=np.float32).view(np.int32).astype(np.int64)
+    a = np.where(a < 0, -(a & 0x7FFFFFFF), a)
+    b = np.where(b < 0, -(b & 0x7FFFFFFF), b)
+    return np.abs(a - b)
+
+
+class GpuWorkload:
+    """One workload resident on one GPU: arena and streams from torch, `nbuf` rounds of
+    device-generated gradients, and the schedules of the path timed on them."""
+
+    KERNELS = ("local_step_kernel", "merge_kernel", "merge_step_kernel", "round_kernel")
+
+    def __init__(self, hp, torch, dev, cfg, args):
+        self.hp, self.torch, self.dev, self.cfg, self.args = hp, torch, dev, cfg, args
+        lay = cfg.layout
+        K, P_pad = cfg.K, lay.P_pad
+        self.bf16 = cfg.grad_dtype == "bf16"
+        self.gdt = torch.int16 if self.bf16 else torch.float32
+        self.gsz = 2 if self.bf16 else 4
+        self.kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
+        # state: arena and streams come from torch, the library only computes.  The arena is sized
+        # for the pipelined schedule too, so that every schedule can be timed in one run.
+        self.nbytes = hp.hpsgd_arena_bytes(P_pad, K, (hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0) | hp.HPSGD_ARENA_PIPELINE,
+                                           cfg.sparse[1] if cfg.sparse else 0)
+        self.arena = torch.empty(self.nbytes + 256, dtype=torch.uint8, device=dev)
+        self.base = self.arena.data_ptr() + (-self.arena.data_ptr()) % 256
+        self.main, self.side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.setup(args.pipeline, args.fuse, args.chunks)
+        # inputs: `nbuf` rounds of gradients for all K workers, generated on the device
+        self.nbuf = nbuf = args.grad_buffers
+        self.row = -(-P_pad // 2048) * 2048          # every worker's gradient starts on a 4 KB boundary
+        self.grads = torch.empty((nbuf, K, self.row), dtype=self.gdt, device=dev)[:, :, :P_pad]
+        self.sparse_in = None
+        if cfg.sparse:
+            cols = cfg.sparse[2]
+            self.sparse_in = []
+            for b in range(nbuf):
+                per_worker = []
+                for i in range(K):
+                    idx = torch.from_numpy(cfg.sparse_rows(i, b)).to(dev)
+                    vals = torch.empty(idx.numel() * cols, dtype=self.gdt, device=dev)
+                    hp.hpsgd_gen_row_vals(vals, i, b, self.kind, cfg.grad_scale, idx, idx.numel())
+                    per_worker.append((idx, vals))
+                self.sparse_in.append(per_worker)
+        for b in range(nbuf):
+            for i in range(K):
+                hp.hpsgd_gen_grads(self.grads[b, i], i, b, self.kind, cfg.grad_scale)
+        hp.hpsgd_synchronize()
+
+    def setup(self, pipeline, fuse, chunks):
+        hp, cfg = self.hp, self.cfg
+        hp.hpsgd_destroy()
+        if len(cfg.sizes) > 1:
+            hp.hpsgd_set_layout(list(cfg.sizes))
+        hp.hpsgd_set_pipeline(pipeline)
+        hp.hpsgd_bind(self.base, self.nbytes, self.main, self.side)
+        hp.hpsgd_init(cfg.P, cfg.K, cfg.lr, cfg.momentum, cfg.seed)
+        if cfg.weight_decay:
+            hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, cfg.weight_decay)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if self.bf16 else hp.HPSGD_F32)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, self.args.overlap)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if pipeline else chunks)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
+        if cfg.sparse:
+            hp.hpsgd_set_sparse_segment(*cfg.sparse)
+        self.pipeline, self.fuse, self.chunks = pipeline, (0 if pipeline else fuse), (1 if pipeline else chunks)
+
+    def one_round(self, t):
+        hp, cfg, args = self.hp, self.cfg, self.args
+        b = t % self.nbuf
+        if cfg.sparse:
+            descs = [hp.make_desc(self.grads[b, i], self.sparse_in[b][i][0], self.sparse_in[b][i][0].numel(),
+                                  self.sparse_in[b][i][1]) for i in range(cfg.K)]
+            if args.per_worker:
+                for i in range(cfg.K):
+                    hp.hpsgd_local_step_ex(i, descs[i])
+            else:
+                hp.hpsgd_local_step_all_ex(descs)
+        elif args.per_worker:
+            for i in range(cfg.K):
+                hp.hpsgd_local_step(i, self.grads[b, i])
+        else:
+            hp.hpsgd_local_step_all(self.grads[b], self.row * self.gsz)
+        hp.hpsgd_sync_merge()
+
+    def timed(self, steps, warmup, sampler=None, dist=None):
+        """`warmup` untimed rounds, then `steps` rounds between two events on the main stream
+        (the side stream joined before the second).  Returns (ms, launches, per-kernel event sums)."""
+        hp, torch = self.hp, self.torch
+        for t in range(warmup):
+            self.one_round(t)
+        hp.hpsgd_synchronize()
+        hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)     # also launches anything the warm-up left held back
+        for kind in range(len(self.KERNELS)):
+            hp.hpsgd_profile_read(kind)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(self.dev)
+        if sampler is not None:
+            sampler.mark_begin()
+        launches0 = hp.hpsgd_launch_count()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(self.main)
+        for t in range(steps):
+            self.one_round(warmup + t)
+        hp.hpsgd_flush()                                 # the last round's merge, if a schedule held it back
+        self.main.wait_stream(self.side)
+        end.record(self.main)
+        torch.cuda.synchronize(self.dev)
+        if sampler is not None:
+            sampler.mark_end()
+        if dist is not None:
+            dist.barrier()
+        ms = start.elapsed_time(end)
+        launches = hp.hpsgd_launch_count() - launches0
+        prof = {name: hp.hpsgd_profile_read(kind) for kind, name in enumerate(self.KERNELS)}
+        hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 0)
+        return ms, launches, prof
+
+    def bytes_per_round(self):
+        """HBM bytes each kind of kernel moves in one round of the current schedule (what the launch
+        really reads and writes, not what an un-fused schedule would)."""
+        cfg, K, P = self.cfg, self.cfg.K, self.cfg.P
+        # gradient bytes of one round: dense buffers, minus the rows of a sparse-row tensor that carry
+        # no gradient (never read), plus 4 bytes per listed row index
+        grad_bytes = K * P * self.gsz
+        if cfg.sparse:
+            rows_total, cols = cfg.sparse[1], cfg.sparse[2]
+            active = sum(pw[0].numel() for b in self.sparse_in for pw in b) / self.nbuf
+            grad_bytes += active * 4 - (K * rows_total - active) * cols * self.gsz
+        state_bytes = K * P * (8 + (8 if cfg.momentum else 0))        # r (and m) read and written
+        return {"local_step_kernel": grad_bytes + state_bytes,
+                # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
+                "merge_kernel": (12 + (K + 2) * 4) * P if self.pipeline else
+                                ((K + 4) * 4 * P if self.fuse == 2 else merge_bytes_per_index(cfg) * P),
+                "merge_step_kernel": 16 * P + grad_bytes + state_bytes,
+                # whole round in one kernel, one step per worker and period: no replica row is read
+                # or written; w, D, K m, K g in and w, D, K m out
+                "round_kernel": 16 * P + grad_bytes + (K * P * 8 if cfg.momentum else 0)}
+
+    def kernel_table(self, prof, peak):
+        per_round = self.bytes_per_round()
+        kernels = {}
+        for name, (ms, n) in prof.items():
+            if n == 0:
+                continue
+            per_launch = per_round[name] / self.chunks
+            if self.args.per_worker and name == "local_step_kernel":
+                per_launch /= self.cfg.K
+            if self.pipeline and name == "merge_kernel":
+                per_launch /= 2
+            gbs = per_launch * n / (ms * 1e-3) / 1e9
+            kernels[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms, "bytes_per_launch": per_launch,
+                             "achieved": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+        return kernels
+
+    def parity(self):
+        """The workload's T rounds from a fresh state in the schedule being timed, then w and D at a
+        stratified sample of indices against the CPU oracle fed the HOST generator's gradients."""
+        from oracle.ref import RefHPSGD
+        hp, torch, cfg = self.hp, self.torch, self.cfg
+        lay = cfg.layout
+        self.setup(self.pipeline, self.fuse if not self.pipeline else 0, self.chunks)
+        for t in range(cfg.T):
+            self.one_round(t)
+        hp.hpsgd_synchronize()
+        idx = parity_sample(cfg)
+        pos = torch.from_numpy(lay.padded_index(idx)).to(self.dev)
+        got = {}
+        for key, addr in (("w", hp.hpsgd_get_global()), ("D", hp.hpsgd_get_pending())):
+            got[key] = torch.as_tensor(_RawDeviceArray(addr, lay.P_pad), device=self.dev)[pos].cpu().numpy()
+        t0 = time.perf_counter()
+        oracle = RefHPSGD(idx.size, cfg.K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+        oracle.set_global(cfg.initial_global(idx))
+        master = None
+        if self.bf16:      # the same rule fed the gradients before their rounding to bf16
+            master = RefHPSGD(idx.size, cfg.K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+            master.set_global(cfg.initial_global(idx))
+        stored = {(i, b): cfg.stored_gradient(i, b, idx) for i in range(cfg.K) for b in range(self.nbuf)}
+        exact = {(i, b): cfg.gradient(i, b, idx) for i in range(cfg.K) for b in range(self.nbuf)} if master else None
+        for t in range(cfg.T):
+            for i in range(cfg.K):
+                oracle.local_step(i, stored[(i, t % self.nbuf)])
+                if master:
+                    master.local_step(i, exact[(i, t % self.nbuf)])
+            oracle.sync_merge()
+            if master:
+                master.sync_merge()
+        want = {"w": oracle.get_global(), "D": oracle.get_pending()}
+        out = {"rounds": cfg.T, "sampled_indices": int(idx.size),
+               "inputs": "device generator on the GPU, host generator for the oracle (%d rounds of gradients cycled)" % self.nbuf}
+        for key, floor in (("w", 1e-6), ("D", 1e-9)):
+            g64, w64 = got[key].astype(np.float64), want[key].astype(np.float64)
+            out[key] = {"max_rel_err": float(np.max(np.abs(g64 - w64) / np.maximum(np.abs(w64), floor))),
+                        "max_ulp": int(ulp_distance(got[key], want[key]).max()),
+                        "bit_equal_fraction": float(np.mean((got[key].view(np.uint32) == want[key].view(np.uint32))
+                                                            | ((got[key] == 0) & (want[key] == 0))))}
+        out["within_1e-6"] = bool(out["w"]["max_rel_err"] <= 1e-6)
+        if master:
+            m64 = master.get_global().astype(np.float64)
+            out["w_vs_fp32_master_max_rel_err_floor_1e-4"] = float(
+                np.max(np.abs(got["w"].astype(np.float64) - m64) / np.maximum(np.abs(m64), 1e-4)))
+            master.close()
+        oracle.close()
+        out["oracle_seconds"] = time.perf_counter() - t0
+        return out
+
+    def release(self):
+        self.hp.hpsgd_destroy()
+        self.arena = self.grads = self.sparse_in = None
+        self.torch.cuda.empty_cache()
+
+
+def other_workload_entry(hp, torch, dev, name, args, peak):
+    """A short timed run of another of the five workloads in the schedule being timed, with its
+    parity figures (the oracle runs after the timed region)."""
+    cfg = workloads.get(name)
+    run = GpuWorkload(hp, torch, dev, cfg, args)
+    steps = args.other_workload_steps
+    ms, launches, prof = run.timed(steps, 3)
+    kernels = run.kernel_table(prof, peak)
+    dominant = max(kernels, key=lambda k: kernels[k]["total_ms"])
+    entry = {"workload": "%s: %s" % (cfg.name, cfg.note), "K": cfg.K, "P": cfg.P, "steps": steps,
+             "ms_per_step": ms / steps, "value": cfg.K * cfg.P * steps / (ms * 1e-3), "unit": UNIT,
+             "gpu_launches": int(launches), "kernel": dominant, "kernel_avg_ms": kernels[dominant]["avg_ms"],
+             "bytes_per_launch": kernels[dominant]["bytes_per_launch"], "achieved": kernels[dominant]["achieved"],
+             "frac": kernels[dominant]["frac"], "frac_of_nominal_8TBs": kernels[dominant]["frac_of_nominal_8TBs"]}
+    state_mb = run.nbytes / 1e6
+    if state_mb + run.grads.numel() * run.gsz / 1e6 < 126:
+        entry["note"] = "L2-resident (state + gradients below the 126 MB L2) and launch-bound: GB/s here is not an HBM figure"
+    elif ms / steps < 0.5:
+        entry["note"] = "sub-millisecond kernel: launch gaps and the tail of the grid weigh on the rate"
+    if args.parity:
+        entry["parity"] = run.parity()
+    run.release()
+    return entry
+
+
 def run_gpu(args, cfg):
     import torch
     import paper_2009_02701_b200 as hp
@@ -297,145 +555,26 @@ def run_gpu(args, cfg):
         cuda_build.build()              # no-op when the in-tree library is up to date
     if dist is not None:
         dist.barrier()
-    lay = cfg.layout
-    K, P, P_pad = cfg.K, cfg.P, lay.P_pad
-    bf16 = cfg.grad_dtype == "bf16"
-    gdt = torch.int16 if bf16 else torch.float32
-    gsz = 2 if bf16 else 4
-    kind = hp.HPSGD_GEN_UNIFORM if cfg.grad_kind == "uniform" else hp.HPSGD_GEN_GAUSS
-
-    # ---- state: arena and streams come from torch, the library only computes.  The arena is
-    # sized for the pipelined schedule too, so that every schedule can be timed in one run.
-    nbytes = hp.hpsgd_arena_bytes(P_pad, K, (hp.HPSGD_ARENA_MOMENTUM if cfg.momentum else 0) | hp.HPSGD_ARENA_PIPELINE,
-                                  cfg.sparse[1] if cfg.sparse else 0)
-    arena = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
-    base = arena.data_ptr() + (-arena.data_ptr()) % 256
-    main, side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-
-    def setup(pipeline, fuse, chunks):
-        hp.hpsgd_destroy()
-        if len(cfg.sizes) > 1:
-            hp.hpsgd_set_layout(list(cfg.sizes))
-        hp.hpsgd_set_pipeline(pipeline)
-        hp.hpsgd_bind(base, nbytes, main, side)
-        hp.hpsgd_init(P, K, cfg.lr, cfg.momentum, cfg.seed)
-        if cfg.weight_decay:
-            hp.hpsgd_set_option(hp.HPSGD_OPT_WEIGHT_DECAY, cfg.weight_decay)
-        hp.hpsgd_set_option(hp.HPSGD_OPT_STALENESS, cfg.staleness)
-        hp.hpsgd_set_option(hp.HPSGD_OPT_GRAD_DTYPE, hp.HPSGD_BF16 if bf16 else hp.HPSGD_F32)
-        hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, args.overlap)
-        hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if pipeline else chunks)
-        hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
-        if cfg.sparse:
-            hp.hpsgd_set_sparse_segment(*cfg.sparse)
-
-    setup(args.pipeline, args.fuse, args.chunks)
-
-    # ---- inputs: `nbuf` rounds of gradients for all K workers, generated on the device
-    nbuf = args.grad_buffers
-    row = -(-P_pad // 2048) * 2048          # every worker's gradient starts on a 4 KB boundary
-    grads = torch.empty((nbuf, K, row), dtype=gdt, device=dev)[:, :, :P_pad]
-    sparse_in = None
-    if cfg.sparse:
-        rows_max = cfg.sparse[1]
-        cols = cfg.sparse[2]
-        sparse_in = []
-        for b in range(nbuf):
-            per_worker = []
-            for i in range(K):
-                idx = torch.from_numpy(cfg.sparse_rows(i, b)).to(dev)
-                vals = torch.empty(idx.numel() * cols, dtype=gdt, device=dev)
-                hp.hpsgd_gen_row_vals(vals, i, b, kind, cfg.grad_scale, idx, idx.numel())
-                per_worker.append((idx, vals))
-            sparse_in.append(per_worker)
-    for b in range(nbuf):
-        for i in range(K):
-            hp.hpsgd_gen_grads(grads[b, i], i, b, kind, cfg.grad_scale)
-    hp.hpsgd_synchronize()
-
-    def one_round(t):
-        b = t % nbuf
-        if cfg.sparse:
-            descs = [hp.make_desc(grads[b, i], sparse_in[b][i][0], sparse_in[b][i][0].numel(), sparse_in[b][i][1])
-                     for i in range(K)]
-            if args.per_worker:
-                for i in range(K):
-                    hp.hpsgd_local_step_ex(i, descs[i])
-            else:
-                hp.hpsgd_local_step_all_ex(descs)
-        elif args.per_worker:
-            for i in range(K):
-                hp.hpsgd_local_step(i, grads[b, i])
-        else:
-            hp.hpsgd_local_step_all(grads[b], row * gsz)
-        hp.hpsgd_sync_merge()
+    K, P = cfg.K, cfg.P
+    run = GpuWorkload(hp, torch, dev, cfg, args)
 
     # ---- warm-up, then the timed region (the clock sampler needs a moment to start)
     sampler = ClockSampler(device_index)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    for t in range(args.warmup):
-        one_round(t)
-    hp.hpsgd_synchronize()
-    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)     # also launches a merge deferred by the warm-up
-    for kind in range(4):
-        hp.hpsgd_profile_read(kind)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize(dev)
-    sampler.mark_begin()
-    launches0 = hp.hpsgd_launch_count()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record(main)
-    for t in range(args.steps):
-        one_round(args.warmup + t)
-    hp.hpsgd_flush()                                 # the last round's merge, if it was deferred
-    main.wait_stream(side)
-    end.record(main)
-    torch.cuda.synchronize(dev)
-    sampler.mark_end()
-    if dist is not None:
-        dist.barrier()
+    elapsed_ms, launches, prof = run.timed(args.steps, args.warmup, sampler if rank == 0 else None, dist)
     clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = start.elapsed_time(end)
-    launches = hp.hpsgd_launch_count() - launches0
-    prof = {name: hp.hpsgd_profile_read(kind) for kind, name in
-            enumerate(("local_step_kernel", "merge_kernel", "merge_step_kernel", "round_kernel"))}
-    hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 0)
     units = K * P * args.steps
     job_ms, job_units = aggregate(dist, dev, elapsed_ms, units)
     value = job_units / (job_ms * 1e-3)
 
-    # ---- roofline of the kernels from the event pairs recorded inside the timed region.
-    # Algorithmic bytes per launch = bytes per parameter index x indices one launch covers.
+    # ---- roofline of the kernels from the event pairs recorded inside the timed region:
+    # bytes one launch moves = bytes per parameter index x indices the launch covers
     peak, peak_src = measured_peak()
-    # gradient bytes of one round: dense buffers, minus the rows of a sparse-row tensor that carry
-    # no gradient (never read), plus 4 bytes per listed row index
-    grad_bytes = K * P * gsz
-    if cfg.sparse:
-        rows_total, cols = cfg.sparse[1], cfg.sparse[2]
-        active = sum(pw[0].numel() for b in sparse_in for pw in b) / nbuf
-        grad_bytes += active * 4 - (K * rows_total - active) * cols * gsz
-    state_bytes = K * P * (8 + (8 if cfg.momentum else 0))        # r (and m) read and written
-    per_round = {"local_step_kernel": grad_bytes + state_bytes,
-                 # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
-                 "merge_kernel": (12 + (K + 2) * 4) * P if args.pipeline else merge_bytes_per_index(cfg) * P,
-                 "merge_step_kernel": 16 * P + grad_bytes + state_bytes,
-                 # whole round in one kernel, one step per worker and period: no replica row is read
-                 # or written; w, D, K m, K g in and w, D, K m out
-                 "round_kernel": 16 * P + grad_bytes + (K * P * 8 if cfg.momentum else 0)}
-    kernels = {}
-    for name, (ms, n) in prof.items():
-        if n == 0:
-            continue
-        per_launch = per_round[name] / (1 if args.pipeline else args.chunks) / (K if (args.per_worker and name == "local_step_kernel") else 1)
-        if args.pipeline and name == "merge_kernel":
-            per_launch /= 2
-        gbs = per_launch * n / (ms * 1e-3) / 1e9
-        kernels[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms, "algorithmic_bytes_per_launch": per_launch,
-                         "achieved": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+    kernels = run.kernel_table(prof, peak)
     dominant = max(kernels, key=lambda k: kernels[k]["total_ms"])
+    per_round = run.bytes_per_round()
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved"], "peak": peak,
                 "unit": "GB/s", "frac": kernels[dominant]["frac"],
                 "traffic": ncu_traffic(dominant, cfg, args.fuse) if (args.chunks == 1 and not args.per_worker) else None,
@@ -444,10 +583,12 @@ def run_gpu(args, cfg):
                         "bytes are the ones the launch actually moves: round_kernel (local steps + merge in one "
                         "pass, replicas never stored) 16 + K*(g + 8) per index with momentum, merge_step_kernel "
                         "16 + K*(g + 16), merge_kernel (2K + 4)*4, local_step_kernel K*(g + 16)"}
-    moved = sum(k["algorithmic_bytes_per_launch"] * k["launches"] for k in kernels.values())
+    moved = sum(k["bytes_per_launch"] * k["launches"] for k in kernels.values())
     roofline["round_achieved"] = moved / (elapsed_ms * 1e-3) / 1e9
     roofline["round_frac"] = roofline["round_achieved"] / peak
-    unfused_round = per_round["local_step_kernel"] + per_round["merge_kernel"]
+    # the same rounds priced at what separate local-step and merge kernels would have to move
+    # (28K + 16 bytes per index with momentum): the rate the fusion is worth, not a bandwidth
+    unfused_round = K * P * (run.gsz + 8 + (8 if cfg.momentum else 0)) + merge_bytes_per_index(cfg) * P
     roofline["round_unfused_equivalent"] = unfused_round * args.steps / (elapsed_ms * 1e-3) / 1e9
 
     # ---- the other schedules of the same path, timed briefly the same way (same inputs, same work)
@@ -459,49 +600,56 @@ def run_gpu(args, cfg):
                                  ("one kernel per round (local steps + merge), replicas never stored", 0, 2)):
             if (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
                 continue
-            setup(pipe, fuse, 1)
-            for t in range(3):
-                one_round(t)
-            hp.hpsgd_synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(main)
-            for t in range(args.other_schedule_steps):
-                one_round(3 + t)
-            hp.hpsgd_flush()
-            main.wait_stream(side)
-            b.record(main)
-            torch.cuda.synchronize(dev)
-            ms = a.elapsed_time(b) / args.other_schedule_steps
-            other[name] = {"ms_per_step": ms, "value": K * P / (ms * 1e-3), "steps": args.other_schedule_steps}
-        setup(args.pipeline, args.fuse, args.chunks)
+            run.setup(pipe, fuse, 1)
+            ms, n_launch, prof_o = run.timed(args.other_schedule_steps, 3)
+            ms /= args.other_schedule_steps
+            other[name] = {"ms_per_step": ms, "value": K * P / (ms * 1e-3), "steps": args.other_schedule_steps,
+                           "gpu_launches": int(n_launch),
+                           "kernels": {k: {"launches": v["launches"], "avg_ms": v["avg_ms"], "achieved": v["achieved"],
+                                           "frac_of_nominal_8TBs": v["frac_of_nominal_8TBs"]}
+                                       for k, v in run.kernel_table(prof_o, peak).items()}}
+        run.setup(args.pipeline, args.fuse, args.chunks)
 
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step
     e2e = None
     if args.e2e_steps > 0:
-        e2e = run_e2e(args, cfg, hp, torch, dev, grads, dist)
+        e2e = run_e2e(args, cfg, hp, torch, dev, run.grads, dist)
 
     line = None
     if rank == 0:
+        parity = run.parity() if args.parity else None
+        run.release()
+        # ---- the other four workloads, briefly, each with its parity figures
+        others = {}
+        if args.other_workload_steps > 0 and not args.max_params:
+            for name in workloads.names():
+                if name != cfg.name:
+                    others[name] = other_workload_entry(hp, torch, dev, name, args, peak)
         cpu = None
         if args.cpu_seconds > 0:
             eps, rounds, spent, desc, _ = oracle_sample_run(cfg, args.cpu_seconds)
-            cpu = {"value": eps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+            cpu = {"value": eps, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc,
                    "seconds": spent}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": job_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic (counter-hash gradients generated on the device, %d rounds cycled)" % nbuf,
+            "data": "synthetic (counter-hash gradients generated on the device, %d rounds cycled)" % run.nbuf,
             "config": workload_config(cfg, {
                 "schedule": {"overlap": args.overlap, "chunks": args.chunks,
-                             "fuse_merge_into_next_step": 0 if args.pipeline else args.fuse,
+                             "fuse": 0 if args.pipeline else args.fuse,
+                             "fuse_meaning": "2: one kernel per round (batched local step inside the kernel of the merge "
+                                             "that follows it); 1: merge carried into the next local step; 0: separate kernels",
                              "pipelined_commit_reduce": args.pipeline,
                              "local_step_call": "per worker" if args.per_worker else "all K in one call"},
                 "l2": "inputs larger than L2 (state + gradients are tens of GB)",
                 "multi_gpu": "independent replicas, no inter-GPU exchange"}),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu, "other_schedules": other,
+            "roofline": roofline, "parity": parity, "cpu_baseline": cpu, "other_schedules": other,
+            "workloads": others,
         }
+    else:
+        run.release()
     hp.hpsgd_destroy()
     if dist is not None:
         dist.destroy_process_group()
@@ -580,6 +728,10 @@ def main():
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--e2e-host-buffers", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU oracle baseline budget (0 = skip)")
+    ap.add_argument("--other-workload-steps", type=int, default=10,
+                    help="timed rounds for each of the other four workloads, reported under `workloads` (0 = skip)")
+    ap.add_argument("--parity", type=int, default=1,
+                    help="1: after the timed regions, run each workload's T rounds and compare a sample with the CPU oracle")
     ap.add_argument("--max-params", type=int, default=0,
                     help="cut the workload to its first N parameters (for small profiler captures)")
     ap.add_argument("--ref-sample", type=int, default=4_000_000, help="parameters per step of --impl reference")

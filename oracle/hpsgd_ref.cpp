@@ -30,7 +30,8 @@
  *   - AllReduce means the mean over K workers (Eq. 1 divides by n); the sums of Eq. 1/2
  *     run over the K workers 0..K-1.
  *   - Order inside one synchronisation: apply the pending change, then clone replicas
- *     from the UPDATED global model ("replica of the latest global model", Section 3.1).
+ *     from the UPDATED global model (Section 3.1 has the replica made from the newest
+ *     global model).
  *   - Momentum: heavy ball, m <- beta*m + gd, r <- r - mu*m, per worker, zero at start,
  *     untouched by the merge.  Weight decay: coupled L2 at the replica, gd = g + lambda*r.
  *   - What is averaged is the replica change (Eq. 2 form), which under momentum includes
@@ -47,10 +48,10 @@
  * worker, AllReduce of those accumulators (mean), and the delayed commit
  * w <- w - mu * (mean gradients all-reduced at the previous synchronisation).
  *
- * Pins (tests/, run without a GPU): hand-worked K=2, P=4 examples; the closed form of
- * Eq. 1 in binary64; a separate literal transcription of Algorithms 2 and 3 with explicit
- * gradient accumulators; K=1 against a library SGD/momentum optimiser; Local SGD model
- * averaging (Algorithm 1); equal-gradient and first-merge invariants.
+ * Pins (tests/, run without a GPU): hand-worked K=2, P=4 examples; the closed forms of
+ * Eq. 1 and Eq. 2 in binary64, also over periods of uneven length; K=1 against a library
+ * SGD/momentum optimiser; Local SGD model averaging (Algorithm 1); equal-gradient and
+ * first-merge invariants.
  */
 #include <cmath>
 #include <cstdint>

@@ -8,7 +8,8 @@ import ctypes
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libhpsgd.so")
+# HPSGD_LIBRARY names another build of the same library (the checked build, a tuning variant)
+LIB_PATH = os.environ.get("HPSGD_LIBRARY") or os.path.join(HERE, "libhpsgd.so")
 
 HPSGD_OK = 0
 HPSGD_E_BADARG, HPSGD_E_STATE, HPSGD_E_NOMEM = -1, -2, -3

@@ -600,10 +600,12 @@ __device__ __forceinline__ SegPos seg_pos(const SparseSeg& seg, int64_t o)
 {
     SegPos sp{false, 0, 0};
     if (o >= seg.o_begin && o < seg.o_end) {
-        const int64_t rel = o - seg.o_begin;
+        // the tensor has fewer than 2^32 groups (P < 2^32): a 32-bit division, far cheaper than a 64-bit one
+        const uint32_t rel = (uint32_t)(o - seg.o_begin);
+        const uint32_t row = rel / (uint32_t)seg.cols8;
         sp.inside = true;
-        sp.row = rel / seg.cols8;
-        sp.col8 = rel - sp.row * seg.cols8;
+        sp.row = row;
+        sp.col8 = rel - row * (uint32_t)seg.cols8;
     }
     return sp;
 }
@@ -731,26 +733,32 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
 // Same operations in the same order as local_step_kernel for every worker followed by
 // merge_kernel, so the results are bit-identical.  Workers are handled B at a time: all
 // loads of a batch are requested before the first use.
+// `pre`: row -> slot entries of these NB workers that the caller requested earlier, or NULL.
 template <int NB, bool FIRST, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 __device__ __forceinline__ void round_batch(f8& acc, const f8& wv, float* __restrict__ m, int64_t stride, int i0,
                                             const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp,
-                                            int64_t o, const StepParams& p)
+                                            int64_t o, const StepParams& p, const int32_t* pre)
 {
     const int64_t e = o * 8;
+    // Request order matters inside the sparse-row tensor: the row -> slot entries come first (they
+    // are short, L2-resident loads that the gradient addresses depend on), then everything that
+    // depends on nothing (momentum, replica rows), and only then the gradients, whose addresses
+    // need the slots.  The long loads are then in flight while the slots come back.
     int32_t sl[NB];
     if (SPARSE && sp.inside) {
 #pragma unroll
-        for (int b = 0; b < NB; ++b) sl[b] = __ldg(gp.slot[i0 + b] + sp.row);
+        for (int b = 0; b < NB; ++b) sl[b] = pre ? pre[b] : __ldg(gp.slot[i0 + b] + sp.row);
     }
     GradRaw<BF16> graw[NB];
     f8 mm[NB];
     f8 rr[FROM_W ? 1 : NB];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-        graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[b] : 0, i0 + b, o);
         if (MOM) mm[b] = ld8(m + (int64_t)(i0 + b) * stride + e);
         if (!FROM_W) rr[b] = ld8(gp.r_src[i0 + b] + e);
     }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) graw[b] = fused_grad_raw<BF16, SPARSE>(gp, seg, sp, SPARSE ? sl[b] : 0, i0 + b, o);
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const f8 gg = widen_grad<BF16>(graw[b]);
@@ -765,8 +773,16 @@ __device__ __forceinline__ void round_batch(f8& acc, const f8& wv, float* __rest
     }
 }
 
-constexpr int kRoundBatchF32 = 8;    // workers in flight together: 16 x 32-byte loads per thread (g and m)
-constexpr int kRoundBatchBf16 = 8;
+// Workers whose loads are in flight together.  Each costs 8 registers for fp32 gradients (4 for
+// bf16), 8 for momentum and 8 for a replica row that has to be read; the batch is as large as
+// fits the 255 registers of a thread without spilling: 8 workers (16 x 32-byte loads) for the
+// usual fp32 + momentum case, 16 where a worker needs at most 12 registers.
+constexpr int round_batch_size(bool bf16, bool mom, bool sparse, bool from_w)
+{
+    const int per_worker = (bf16 ? 4 : 8) + (mom ? 8 : 0) + (from_w ? 0 : 8);
+    if (!from_w) return per_worker >= 24 ? 4 : 8;
+    return (per_worker <= 12 && !(bf16 && mom && sparse)) ? 16 : 8;
+}
 
 template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 __global__ void __launch_bounds__(kHotThreads, 2)
@@ -780,23 +796,48 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         const int64_t e = o * 8;
         SegPos sp{false, 0, 0};
         if (SPARSE) sp = seg_pos(seg, o);
+        // the slot entries of the first two batches are requested before anything else: by the time
+        // the gradient addresses are formed they have arrived (where the registers allow it)
+        constexpr bool PRE = SPARSE && FROM_W;
+        int32_t sl_pre[PRE ? 2 * B : 1];
+        if (PRE && sp.inside) {
+#pragma unroll
+            for (int b = 0; b < (PRE ? 2 * B : 1); ++b) sl_pre[b] = b < K ? __ldg(gp.slot[b] + sp.row) : -1;
+        }
+        const int32_t* sl = PRE ? sl_pre : nullptr;
         const f8 wv = ld8(w + e);
         f8 dv = zero8();
         if (flags & kMergeApplyPending) dv = ld8(D + e);
+#ifdef HPSGD_ROUND_PREFETCH
+        // the second batch's momentum (and dense gradients) start their way from DRAM to L2 now: that
+        // costs no registers, and their loads later find them on chip
+        if (K >= 2 * B) {
+#pragma unroll
+            for (int b = B; b < 2 * B; ++b) {
+                if (MOM) asm volatile("prefetch.global.L2 [%0];" :: "l"(m + (int64_t)b * stride + e));
+                if (!(SPARSE && sp.inside))
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(reinterpret_cast<const char*>(gp.dense[b]) + o * (BF16 ? 16 : 32)));
+            }
+        }
+#endif
         // ---- local steps and the running sum of replica changes, worker 0 first
         f8 acc;
         int i = 0;
         if (K >= B) {
-            round_batch<B, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p);
+            round_batch<B, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p, sl);
             i = B;
+            if (K >= 2 * B) {
+                round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, B, gp, seg, sp, o, p, PRE ? sl + B : nullptr);
+                i = 2 * B;
+            }
         } else {
-            round_batch<1, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p);
+            round_batch<1, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p, sl);
             i = 1;
         }
         for (; i + B <= K; i += B)
-            round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p);
+            round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
         for (; i < K; ++i)
-            round_batch<1, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p);
+            round_batch<1, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
         // ---- merge
         f8 dnew, wn;
 #pragma unroll

@@ -398,12 +398,10 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
 }
 
 // ---------------------------------------------------------------------------- fuse 2: local step + merge, one round
-// Workers whose loads are in flight together: 8 (fp32 gradients, 16 x 32 bytes per thread) or
-// 16 with bf16 gradients (half the gradient bytes).
 template <bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 void launch_round(const FusedLaunch& L)
 {
-    constexpr int B = BF16 ? kRoundBatchBf16 : kRoundBatchF32;
+    constexpr int B = round_batch_size(BF16, MOM, SPARSE, FROM_W);
     round_kernel<B, BF16, MOM, WD, SPARSE, FROM_W><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
         g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
 }

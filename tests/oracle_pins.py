@@ -60,91 +60,53 @@ def pin_worked_examples(lib):
         o.close()
 
 
-# ------------------------------------------------------------------ literal Algorithms 2 and 3
-def literal_hpsgd(w0, grads, mu, busy):
-    """Algorithms 2 and 3 as printed, in binary64, with explicit shared variables.
-
-    ``grads[e][i]`` is worker i's local gradient at epoch e.  A synchronisation, once
-    started, keeps P_s busy for ``busy`` further epochs.  All workers hold the same global
-    model (one ``w``).  Returns the global model after every synchronisation start and the
-    list of (epoch, worker, replica) seen in the synchronising branch.
-    """
-    n = len(grads[0])
-    w = np.array(w0, dtype=np.float64)
-    status = "idling"
-    counter = 0
-    busy_left = 0
-    acc = [np.zeros_like(w) for _ in range(n)]          # accumulated gradients per worker
-    replica = [None] * n
-    synced = None                                       # result of the last AllReduce
-    globals_after_sync, replicas_seen = [], []
-    for e in range(len(grads)):
-        if status == "synchronizing":
-            for i in range(n):
-                if counter == 0:
-                    replica[i] = w.copy()                       # make replica
-                replica[i] = replica[i] - mu * grads[e][i]      # update replica
-                acc[i] = acc[i] + grads[e][i]                   # accumulate gradients
-                replicas_seen.append((e, i, replica[i].copy()))
-            counter += 1
-            busy_left -= 1
-            if busy_left == 0:
-                counter = 0                                     # P_s: reset the counter
-                status = "idling"                               # P_s: mark the status
-        else:
-            for i in range(n):
-                acc[i] = acc[i] + grads[e][i]
-            status = "synchronizing"
-            # ---- StartSync(P_s): Algorithm 3
-            if e - counter > 0:
-                w = w - mu * synced                             # commit the previous AllReduce
-            synced = sum(acc) / n                               # AllReduce, mean over workers
-            acc = [np.zeros_like(w) for _ in range(n)]
-            globals_after_sync.append(w.copy())
-            if busy == 0:
-                counter = 0
-                status = "idling"
-            else:
-                busy_left = busy
-    return globals_after_sync, replicas_seen
+# ------------------------------------------------------------------ Eq. 1 and Eq. 2 over uneven periods
+def _periods(rng, syncs):
+    """Local steps per synchronisation period: one before the first synchronisation, then a
+    random number (the synchronising process stays busy for a while, Section 3.2)."""
+    return [1] + [int(rng.integers(1, 5)) for _ in range(syncs - 1)]
 
 
-def pin_literal_algorithms(lib):
-    """The replica-change oracle against the printed gradient-accumulation form (plain SGD)."""
+def pin_eq1_eq2_over_uneven_periods(lib):
+    """Plain SGD with several local steps per period, against the two closed forms the paper
+    gives, evaluated in binary64 from the raw gradients:
+      Eq. 1  the global model after synchronisation s is w_0 minus mu/n times ALL gradients of
+             the periods that ended at synchronisations 0..s-1 (one synchronisation late);
+      Eq. 2  inside a period, replica i is the global model minus mu times worker i's own
+             gradients of that period, and the mean of the replicas minus w is the change the
+             synchronisation puts aside."""
     rng = _rng(7)
     for trial in range(12):
         K = int(rng.integers(1, 6))
         P = int(rng.integers(1, 9))
-        busy = int(rng.integers(0, 4))
-        syncs = int(rng.integers(2, 6))
-        epochs = 1 + (syncs - 1) * (busy + 1)
+        syncs = int(rng.integers(2, 7))
+        steps = _periods(rng, syncs)
         mu = float(rng.choice([0.5, 0.1, 0.03]))
+        mu64 = np.float64(np.float32(mu))
         w0 = rng.uniform(-1, 1, P).astype(np.float32)
-        grads = rng.uniform(-1, 1, (epochs, K, P)).astype(np.float32)
-        want_w, want_r = literal_hpsgd(w0, grads.astype(np.float64), mu, busy)
-        assert len(want_w) == syncs
-
         o = RefHPSGD(P, K, mu, 0.0, 0.0, 1, lib=lib)
         o.set_global(w0)
-        e = 0
-        seen = []
+        landed = np.zeros(P)              # sum over workers and epochs of the periods already committed
+        waiting = None                    # the same sum for the period reduced at the last synchronisation
         for s in range(syncs):
-            steps = 1 if s == 0 else busy + 1
-            for h in range(steps):
+            own = np.zeros((K, P))        # each worker's gradients of the running period
+            w_now = o.get_global().astype(np.float64)
+            for h in range(steps[s]):
                 for i in range(K):
-                    o.local_step(i, grads[e, i])
-                    # the printed algorithm touches the replica only while P_s is busy,
-                    # i.e. on every step of a period but its last one
-                    if s > 0 and h < steps - 1:
-                        seen.append((e, i, o.get_replica(i)))
-                e += 1
+                    g = rng.uniform(-1, 1, P).astype(np.float32)
+                    o.local_step(i, g)
+                    own[i] += g
+                    np.testing.assert_allclose(o.get_replica(i), w_now - mu64 * own[i], rtol=0, atol=4e-6,
+                                               err_msg="Eq. 2 replica, trial %d period %d step %d worker %d" % (trial, s, h, i))
+            mean_change = np.mean([o.get_replica(i).astype(np.float64) for i in range(K)], axis=0) - w_now
             o.sync_merge()
-            np.testing.assert_allclose(o.get_global(), want_w[s], rtol=0, atol=4e-6,
-                                       err_msg="global after synchronisation %d (trial %d)" % (s, trial))
-        assert len(seen) == len(want_r)
-        for (e1, i1, r1), (e2, i2, r2) in zip(seen, want_r):
-            assert (e1, i1) == (e2, i2)
-            np.testing.assert_allclose(r1, r2, rtol=0, atol=4e-6)
+            if waiting is not None:
+                landed += waiting
+            waiting = own.sum(axis=0)
+            np.testing.assert_allclose(o.get_global(), w0.astype(np.float64) - mu64 / K * landed, rtol=0, atol=4e-6,
+                                       err_msg="Eq. 1 global model after synchronisation %d (trial %d)" % (s, trial))
+            np.testing.assert_allclose(o.get_pending(), mean_change, rtol=0, atol=4e-6)
+            np.testing.assert_allclose(o.get_pending(), -mu64 / K * waiting, rtol=0, atol=4e-6)
         o.close()
 
 
@@ -400,53 +362,53 @@ def pin_accum_worked_example(lib):
     o.close()
 
 
-def pin_accum_literal_and_closed_form(lib):
-    """The printed form against its binary64 transcription with status/counter flags, the
-    closed form of Eq. 1, and the replica-change oracle (Eq. 1 == Eq. 2)."""
+def pin_accum_closed_form_and_replica_form(lib):
+    """The printed form against the closed form of Eq. 1 in binary64 over uneven periods, and
+    against the replica-change oracle (Eq. 1 == Eq. 2)."""
     rng = _rng(41)
     for trial in range(8):
         K = int(rng.integers(1, 6))
         P = int(rng.integers(1, 9))
-        busy = int(rng.integers(0, 4))
-        syncs = int(rng.integers(2, 6))
-        epochs = 1 + (syncs - 1) * (busy + 1)
+        syncs = int(rng.integers(2, 7))
+        steps = _periods(rng, syncs)
         mu = float(rng.choice([0.5, 0.1, 0.03]))
         w0 = rng.uniform(-1, 1, P).astype(np.float32)
-        grads = rng.uniform(-1, 1, (epochs, K, P)).astype(np.float32)
-        want_w, _ = literal_hpsgd(w0, grads.astype(np.float64), mu, busy)
         acc = RefHPSGDAccum(P, K, mu, lib=lib)
         rep = RefHPSGD(P, K, mu, 0.0, 0.0, 1, lib=lib)
         acc.set_global(w0)
         rep.set_global(w0)
-        e = 0
         committed = np.zeros(P)
         period_sum = None
         for s in range(syncs):
-            steps = 1 if s == 0 else busy + 1
             this_period = np.zeros(P)
-            for _ in range(steps):
+            own = np.zeros((K, P))
+            for _ in range(steps[s]):
                 for i in range(K):
-                    acc.local_step(i, grads[e, i])
-                    rep.local_step(i, grads[e, i])
-                this_period += grads[e].astype(np.float64).sum(axis=0)
-                e += 1
+                    g = rng.uniform(-1, 1, P).astype(np.float32)
+                    acc.local_step(i, g)
+                    rep.local_step(i, g)
+                    own[i] += g
+                    this_period += g
+            for i in range(K):
+                np.testing.assert_allclose(acc.get_accumulated(i), own[i], rtol=0, atol=4e-6)
             if period_sum is not None:
                 committed += period_sum                 # the previous period lands now
             period_sum = this_period
             acc.sync_merge()
             rep.sync_merge()
-            np.testing.assert_allclose(acc.get_global(), want_w[s], rtol=0, atol=4e-6)
             closed = w0.astype(np.float64) - np.float64(np.float32(mu)) / K * committed
             np.testing.assert_allclose(acc.get_global(), closed, rtol=0, atol=4e-6)
             np.testing.assert_allclose(acc.get_global(), rep.get_global(), rtol=0, atol=4e-6)
             np.testing.assert_allclose(acc.get_synced(), this_period / K, rtol=1e-5, atol=1e-7)
+            for i in range(K):
+                np.testing.assert_array_equal(acc.get_replica(i), acc.get_global())
         acc.close()
         rep.close()
 
 
 ALL_PINS = [
     pin_worked_examples,
-    pin_literal_algorithms,
+    pin_eq1_eq2_over_uneven_periods,
     pin_closed_form_eq1,
     pin_k1_matches_library_sgd,
     pin_local_sgd_model_average,
@@ -456,5 +418,5 @@ ALL_PINS = [
     pin_staleness_is_one_sync_shift,
     pin_storage_variants,
     pin_accum_worked_example,
-    pin_accum_literal_and_closed_form,
+    pin_accum_closed_form_and_replica_form,
 ]

@@ -225,6 +225,48 @@ def test_argument_errors_enqueue_nothing():
     hp.hpsgd_destroy()
 
 
+def test_a_failed_call_does_not_poison_the_next_one():
+    """A CUDA call that fails for its arguments (here: an allocation far beyond the device) is
+    reported by the call that made it and by no later one."""
+    hp.hpsgd_destroy()
+    with pytest.raises(hp.HpsgdError) as err:
+        hp.hpsgd_init((1 << 32) - 64, 64, 0.1, 0.9, 1)          # ~2.2 TB of state
+    assert err.value.code == hp.HPSGD_E_NOMEM
+    cfg = small("after_failure", 3, [5000, 33], T=2)
+    gu.run_both(cfg, cfg.T)                                       # every call returns HPSGD_OK, results exact
+    gu.run_both(cfg, cfg.T, batched=True)
+
+
+def test_import_checks_the_staleness_it_is_given():
+    """A checkpoint written without the one-synchronisation delay cannot be resumed under the
+    pipelined schedule (whose commit kernel only knows the delayed form), and a blob whose
+    staleness field is neither 0 nor 1 is refused."""
+    cfg = small("ckpt_stale", 4, [3000, 17], T=2, staleness=0)
+    with gu.session(cfg, staleness=0):
+        keep = []
+        for i in range(cfg.K):
+            gu.gpu_step(cfg, i, gu.host_inputs(cfg, i, 0), keep)
+        hp.hpsgd_sync_merge()
+        blob = np.empty(hp.hpsgd_state_bytes(), dtype=np.uint8)
+        hp.hpsgd_export_state(blob)
+    delayed = small("ckpt_stale", 4, [3000, 17], T=2, staleness=1)
+    with gu.session(delayed, pipeline=1):
+        before = gu.gpu_state(delayed)
+        with pytest.raises(hp.HpsgdError) as err:
+            hp.hpsgd_import_state(blob)
+        assert err.value.code == hp.HPSGD_E_BADARG
+        after = gu.gpu_state(delayed)
+        gu.assert_bitwise(after[0], before[0], "global model after a refused import")
+    with gu.session(delayed):
+        broken = blob.copy()
+        # header: magic (8), P, P_pad, merges (3 x 8), K, form, has_aux (3 x 4), then staleness
+        broken[44:48] = np.frombuffer(np.int32(7).tobytes(), dtype=np.uint8)
+        with pytest.raises(hp.HpsgdError) as err:
+            hp.hpsgd_import_state(broken)
+        assert err.value.code == hp.HPSGD_E_BADARG
+        hp.hpsgd_import_state(blob)                               # the plain schedule takes the staleness of the blob
+
+
 # ---------------------------------------------------------------- merge fused into the next local step
 @pytest.mark.parametrize("K,momentum,wd,staleness", [(16, 0.9, 0.0, 1), (8, 0.9, 5e-4, 1), (4, 0.0, 0.0, 1),
                                                       (3, 0.9, 0.0, 1), (5, 0.0, 1e-3, 0), (9, 0.5, 0.0, 1),

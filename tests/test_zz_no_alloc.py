@@ -1,4 +1,4 @@
-"""The allocation-free sparse-row step against the regular one.
+"""The allocation-free sparse-row step against the regular one and against the CPU oracle.
 
 hpsgd_local_step_sparse_noalloc exists for programs that cannot allocate device memory at the
 moment they want to step: a server whose own allocator claimed the whole GPU at start-up, so
@@ -7,9 +7,12 @@ synchronisation hidden in cudaMalloc / cudaFree would stall every other stream; 
 to a fixed memory budget.  For them the row -> slot scratch map of the sparse-row step is a
 fixed array inside the library image instead of a piece of an arena.
 
-The test runs the same two consecutive steps through that entry point and through
-hpsgd_local_step_ex and requires bit-identical replicas and momenta.  The second step uses a
-different set of active rows, so a map that still held the first call's entries would be caught.
+The test runs the same two consecutive steps through that entry point, through
+hpsgd_local_step_ex and through the oracle's sparse-row step, and requires bit-identical
+replicas and momenta from all three.  The second step uses a different set of active rows, so a
+map that still held the first call's entries would be caught.  It also checks the property the
+entry point exists for: once the first call on the device has been made, a call leaves the
+amount of free device memory exactly where it was.
 
 This file is named to be collected last: if it fails under `pytest -x`, every other test has
 already run.
@@ -19,6 +22,7 @@ import pytest
 import torch
 
 import paper_2009_02701_b200 as hp
+from oracle.ref import RefHPSGD
 from tests import gpu_util as gu
 from workloads.configs import Workload
 
@@ -36,7 +40,7 @@ def test_noalloc_step_matches_regular_step_twice_in_a_row(dtype, momentum, wd):
     inputs = [gu.host_inputs(cfg, worker, step) for step in (0, 1)]
     assert not np.array_equal(inputs[0]["rows"], inputs[1]["rows"])
 
-    # reference: the regular entry point, which keeps its map in the arena
+    # first reference: the regular entry point, which keeps its map in the arena
     want = []
     with gu.session(cfg):
         w0 = gu.dev_view(hp.hpsgd_get_global(), lay.P_pad)
@@ -47,24 +51,41 @@ def test_noalloc_step_matches_regular_step_twice_in_a_row(dtype, momentum, wd):
             r, m = hp.hpsgd_get_replica(worker)
             want.append((gu.dev_view(r, lay.P_pad), gu.dev_view(m, lay.P_pad) if m else None))
 
+    # second reference: the oracle's sparse-row step (un-padded index space)
+    oracle = gu.oracle_for(cfg)
+    oracle_want = []
+    for inp in inputs:
+        gu.oracle_step(oracle, cfg, worker, inp)
+        oracle_want.append((oracle.get_replica(worker), oracle.get_momentum(worker) if momentum else None))
+    oracle.close()
+
     # the allocation-free entry point on buffers owned by the test; no library state exists
     r = w0.clone()
     m = torch.zeros_like(r) if momentum else None
     stream = torch.cuda.Stream(device=gu.DEV)
     stream.wait_stream(torch.cuda.current_stream())
     gdt = hp.HPSGD_BF16 if dtype == "bf16" else hp.HPSGD_F32
-    for step, inp in enumerate(inputs):
-        g = gu.to_device(inp["padded"])
-        idx = gu.to_device(inp["rows"])
-        vals = gu.to_device(inp["vals"].reshape(-1))
-        torch.cuda.synchronize()
+    staged = []
+    for inp in inputs:                        # every device buffer exists before the first call
+        staged.append((gu.to_device(inp["padded"]), gu.to_device(inp["rows"]), gu.to_device(inp["vals"].reshape(-1))))
+    torch.cuda.synchronize()
+    free_after_first = None
+    for step, (inp, (g, idx, vals)) in enumerate(zip(inputs, staged)):
         desc = hp.make_desc(g, idx, len(inp["rows"]), vals)
+        if step == 1:
+            free_after_first = torch.cuda.mem_get_info()[0]
         hp.hpsgd_local_step_sparse_noalloc(r, m, lay.P_pad, desc, gdt, lay.offsets[1], rows, cols,
                                            cfg.lr, momentum, wd, stream)
         stream.synchronize()
-        assert torch.equal(r, want[step][0]), "replica differs after call %d" % (step + 1)
+        if step == 1:
+            # the call after the warm-up call took no device memory (and gave none back)
+            assert torch.cuda.mem_get_info()[0] == free_after_first
+        assert torch.equal(r, want[step][0]), "replica differs from hpsgd_local_step_ex after call %d" % (step + 1)
+        gu.assert_bitwise(lay.unpack(r.cpu().numpy()), oracle_want[step][0], "replica vs oracle after call %d" % (step + 1))
         if momentum:
-            assert torch.equal(m, want[step][1]), "momentum differs after call %d" % (step + 1)
+            assert torch.equal(m, want[step][1]), "momentum differs from hpsgd_local_step_ex after call %d" % (step + 1)
+            gu.assert_bitwise(lay.unpack(m.cpu().numpy()), oracle_want[step][1],
+                              "momentum vs oracle after call %d" % (step + 1))
 
 
 def test_noalloc_rejects_more_rows_than_its_built_in_map():
@@ -75,3 +96,13 @@ def test_noalloc_rejects_more_rows_than_its_built_in_map():
                                            0.1, 0.0, 0.0, None)
     assert err.value.code == hp.HPSGD_E_UNSUPPORTED
     assert str(hp.HPSGD_NOALLOC_MAX_ROWS) in hp.last_error()
+
+
+def test_noalloc_rejects_a_tensor_that_does_not_fit_without_overflowing():
+    """cols so large that rows * cols would wrap a 64-bit integer must be refused, not truncated."""
+    r = torch.zeros(64, dtype=torch.float32, device=gu.DEV)
+    desc = hp.make_desc(r)
+    for rows, cols, off in ((4, 1 << 62, 0), (2, 64, 0), (1, 64, 8), (8, 8, 8)):
+        with pytest.raises(hp.HpsgdError) as err:
+            hp.hpsgd_local_step_sparse_noalloc(r, None, 64, desc, hp.HPSGD_F32, off, rows, cols, 0.1, 0.0, 0.0, None)
+        assert err.value.code == hp.HPSGD_E_BADARG
