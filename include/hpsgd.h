@@ -67,18 +67,21 @@ enum {
                                       local step (hpsgd_local_step_all[_ex]) both run as ONE kernel in
                                       which the re-cloned replicas never go to memory before they are
                                       stepped; any other call first launches the merge on its own.
-                                   2: one kernel per round.  A batched local step is held back; the
-                                      hpsgd_sync_merge that follows runs it together with the merge: every
-                                      worker is stepped in registers, its change enters the K-way sum, and
-                                      the stepped replica is never stored, because the merge re-clones it
-                                      anyway.  Merges also stop writing the K re-cloned replicas: a replica
+                                   2: one kernel per round.  Local steps are held back (hpsgd_local_step[_ex]
+                                      and the batched calls alike; at most one per worker, all dense or all
+                                      sparse-row); if every worker holds one when hpsgd_sync_merge comes, it
+                                      runs them together with the merge: every worker is stepped in
+                                      registers, its change enters the K-way sum, and the stepped replica is
+                                      never stored, because the merge re-clones it anyway.  Merges also stop writing the K re-cloned replicas: a replica
                                       that nothing has stepped since its clone IS w and is read from w
                                       ("lazy clone"; hpsgd_get_replica then returns w's address).  With one
                                       local step per worker and period no replica row is read or written
                                       at all: per index w, D, K momenta and K gradients come in and w, D,
-                                      K momenta go out.  Any other call first launches a held-back step on
-                                      its own.  The gradients of a held-back step are read when it is
-                                      launched: leave them alone until the next library call returns.
+                                      K momenta go out.  Anything else (a second step of a worker, a merge
+                                      while only some workers hold a step, any other call) first launches
+                                      the held-back steps on their own.  The gradients of a held-back step
+                                      are read when it is launched: leave them alone until hpsgd_sync_merge
+                                      (or hpsgd_flush / hpsgd_synchronize) has returned.
                                    For callers whose gradients are already resident (a simulation, a
                                    benchmark) 2 is the fastest; a trainer that computes the next gradients
                                    while the merge runs wants 0. */

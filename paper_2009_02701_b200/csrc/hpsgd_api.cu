@@ -150,6 +150,7 @@ int hpsgd_init(int64_t P, int K, float lr, float momentum, uint64_t seed)
     g.d_table = reinterpret_cast<int64_t*>(g.arena + a.table);
     g.at_w.assign(K, 1);
     g.row_valid.assign(K, 1);
+    g.step_held.assign(K, 0);
     g.wbuf[0] = g.w;
     g.rbuf[0] = g.r;
     if (g.pipeline) {
@@ -371,9 +372,10 @@ int hpsgd_local_step(int worker, const void* grads)
     TRY(need_init());
     TRY(check_worker(worker));
     TRY(check_grad_ptr(grads, "grads"));
-    TRY(flush_deferred());
     BatchPtrs gp{};
     gp.dense[0] = grads;
+    if (lazy_clones()) return hold_step(worker, gp, 0, false);     // fuse 2: held back for the merge it will run with
+    TRY(flush_deferred());
     return enqueue_local(worker, 1, gp, false);
 }
 
@@ -384,9 +386,12 @@ int hpsgd_local_step_ex(int worker, const hpsgd_grad_desc* desc)
     if (g.sp_tensor < 0) return fail(HPSGD_E_STATE, "no sparse-row tensor declared");
     TRY(check_desc(desc));
     TRY(validate_rows(desc, g.sp_rows, g.main));
-    TRY(flush_deferred());
+    const bool hold = lazy_clones();
+    // a held step of this worker still uses its slot map; held dense steps cannot share a launch with this one
+    if (!hold || (g.steps_held && (g.step_held[worker] || !g.deferred_sparse))) TRY(flush_deferred());
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(worker, 1, desc, &gp));
+    if (hold) return hold_step(worker, gp, 0, true);
     return enqueue_local(worker, 1, gp, true);
 }
 
@@ -403,12 +408,10 @@ int hpsgd_local_step_all(const void* grads, int64_t worker_stride_bytes)
         return enqueue_fused(gp, false);
     }
     TRY(flush_deferred());
-    if (lazy_clones()) {                   // fuse 2: held back for the merge it will run with
-        g.deferred_gp = BatchPtrs{};
-        for (int i = 0; i < g.K; ++i)
-            g.deferred_gp.dense[i] = static_cast<const char*>(grads) + (int64_t)i * worker_stride_bytes;
-        g.deferred_sparse = false;
-        g.step_deferred = true;
+    if (lazy_clones()) {                   // fuse 2: held back for the merge they will run with
+        BatchPtrs gp{};
+        for (int i = 0; i < g.K; ++i) gp.dense[i] = static_cast<const char*>(grads) + (int64_t)i * worker_stride_bytes;
+        for (int i = 0; i < g.K; ++i) TRY(hold_step(i, gp, i, false));
         return HPSGD_OK;
     }
     for (int w0 = 0; w0 < g.K; w0 += kMaxBatch) {
@@ -428,14 +431,12 @@ int hpsgd_local_step_all_ex(const hpsgd_grad_desc* descs)
     if (!descs) return fail(HPSGD_E_BADARG, "descriptor array is NULL");
     for (int i = 0; i < g.K; ++i) TRY(check_desc(descs + i));
     for (int i = 0; i < g.K; ++i) TRY(validate_rows(descs + i, g.sp_rows, g.main));
-    if (g.step_deferred) TRY(flush_deferred());          // an earlier held-back step still uses the slot maps
+    if (g.steps_held) TRY(flush_deferred());             // held-back steps still use the slot maps
     BatchPtrs gp{};
     TRY(enqueue_slot_maps(0, g.K, descs, &gp));
     if (g.merge_deferred) return enqueue_fused(gp, true);
     if (lazy_clones()) {
-        g.deferred_gp = gp;
-        g.deferred_sparse = true;
-        g.step_deferred = true;
+        for (int i = 0; i < g.K; ++i) TRY(hold_step(i, gp, i, true));
         return HPSGD_OK;
     }
     return enqueue_local(0, g.K, gp, true);
@@ -473,7 +474,8 @@ int hpsgd_sync_merge(void)
     else if (g.D_valid) flags |= kMergeApplyPending;
     g.D_valid = true;
     g.merges += 1;
-    if (g.step_deferred) return enqueue_round(flags);    // fuse 2: the held-back step and this merge, one kernel
+    if (g.steps_held == g.K) return enqueue_round(flags);   // fuse 2: every worker's held-back step and this merge, one kernel
+    if (g.steps_held) TRY(flush_deferred());                // some workers only: their steps run first, on their own
     if (g.pipeline) return enqueue_pipelined_merge(flags);
     if (g.fuse == 1 && g.form == HPSGD_FORM_REPLICA_CHANGE) {
         g.merge_deferred = true;
@@ -694,7 +696,7 @@ int64_t hpsgd_tensor_offset(int tensor_id)
 int hpsgd_gen_grads(void* out, int worker, int step, int kind, double scale)
 {
     TRY(check_gen_args(out, worker, step, kind));
-    if (g.step_deferred) TRY(flush_deferred());   // a held-back step may still have to read what `out` holds now
+    if (g.steps_held) TRY(flush_deferred());   // a held-back step may still have to read what `out` holds now
     const GenParams gp = gen_params(worker, step, kind, scale);
     const size_t n = g.sizes.size();
     if (g.grad_dtype == HPSGD_BF16)
@@ -715,7 +717,7 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
     if (n_rows < 0 || n_rows > g.sp_rows) return fail(HPSGD_E_BADARG, "n_rows out of range");
     if (n_rows == 0) return HPSGD_OK;
     if (!row_idx) return fail(HPSGD_E_BADARG, "row_idx is NULL");
-    if (g.step_deferred) TRY(flush_deferred());
+    if (g.steps_held) TRY(flush_deferred());
     const GenParams gp = gen_params(worker, step, kind, scale);
     const int64_t n = (int64_t)n_rows * g.sp_cols;
     if (g.grad_dtype == HPSGD_BF16)

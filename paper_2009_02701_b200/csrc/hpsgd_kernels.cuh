@@ -733,10 +733,11 @@ merge_step_kernel(float* __restrict__ w, float* __restrict__ D, float* __restric
 // Same operations in the same order as local_step_kernel for every worker followed by
 // merge_kernel, so the results are bit-identical.  Workers are handled B at a time: all
 // loads of a batch are requested before the first use.
-// `pre`: row -> slot entries of these NB workers that the caller requested earlier, or NULL.
-template <int NB, bool FIRST, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
-__device__ __forceinline__ void round_batch(f8& acc, const f8& wv, float* __restrict__ m, int64_t stride, int i0,
-                                            const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp,
+// `first`: worker i0 is worker 0, whose change opens the sum.  `pre`: row -> slot entries of these
+// NB workers that the caller requested earlier, or NULL.
+template <int NB, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+__device__ __forceinline__ void round_batch(f8& acc, bool first, const f8& wv, float* __restrict__ m, int64_t stride,
+                                            int i0, const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp,
                                             int64_t o, const StepParams& p, const int32_t* pre)
 {
     const int64_t e = o * 8;
@@ -767,7 +768,7 @@ __device__ __forceinline__ void round_batch(f8& acc, const f8& wv, float* __rest
             const float r_old = FROM_W ? wv.v[q] : rr[FROM_W ? 0 : b].v[q];
             const float r_new = step1<MOM, WD>(gg.v[q], mm[b].v[q], r_old, p);
             const float change = __fsub_rn(r_new, wv.v[q]);
-            acc.v[q] = (FIRST && b == 0) ? change : __fadd_rn(acc.v[q], change);
+            acc.v[q] = (b == 0 && first) ? change : __fadd_rn(acc.v[q], change);
         }
         if (MOM) st8(m + (int64_t)(i0 + b) * stride + e, mm[b]);
     }
@@ -781,7 +782,25 @@ constexpr int round_batch_size(bool bf16, bool mom, bool sparse, bool from_w)
 {
     const int per_worker = (bf16 ? 4 : 8) + (mom ? 8 : 0) + (from_w ? 0 : 8);
     if (!from_w) return per_worker >= 24 ? 4 : 8;
-    return (per_worker <= 12 && !(bf16 && mom && sparse)) ? 16 : 8;
+    if (sparse && (mom || !bf16)) return 8;          // the slot entries requested ahead take registers too
+    return per_worker <= 12 ? 16 : 8;
+}
+
+// Workers [i, K) that do not fill a whole batch: one batch of NB if that many are left, then the
+// same with half of it, down to one worker, so that a remainder of n workers takes about log2(n)
+// rounds of loads instead of n.
+template <int NB, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+__device__ __forceinline__ void round_rest(f8& acc, int& i, int K, const f8& wv, float* __restrict__ m, int64_t stride,
+                                           const BatchPtrs& gp, const SparseSeg& seg, const SegPos& sp, int64_t o,
+                                           const StepParams& p)
+{
+    if constexpr (NB >= 1) {
+        if (i + NB <= K) {
+            round_batch<NB, BF16, MOM, WD, SPARSE, FROM_W>(acc, i == 0, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
+            i += NB;
+        }
+        round_rest<NB / 2, BF16, MOM, WD, SPARSE, FROM_W>(acc, i, K, wv, m, stride, gp, seg, sp, o, p);
+    }
 }
 
 template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
@@ -800,7 +819,7 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         // the gradient addresses are formed they have arrived (where the registers allow it)
         constexpr bool PRE = SPARSE && FROM_W;
         int32_t sl_pre[PRE ? 2 * B : 1];
-        if (PRE && sp.inside) {
+        if (PRE && sp.inside && K >= B) {
 #pragma unroll
             for (int b = 0; b < (PRE ? 2 * B : 1); ++b) sl_pre[b] = b < K ? __ldg(gp.slot[b] + sp.row) : -1;
         }
@@ -819,20 +838,16 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         f8 acc;
         int i = 0;
         if (K >= B) {
-            round_batch<B, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p, sl);
+            round_batch<B, BF16, MOM, WD, SPARSE, FROM_W>(acc, true, wv, m, stride, 0, gp, seg, sp, o, p, sl);
             i = B;
             if (K >= 2 * B) {
-                round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, B, gp, seg, sp, o, p, PRE ? sl + B : nullptr);
+                round_batch<B, BF16, MOM, WD, SPARSE, FROM_W>(acc, false, wv, m, stride, B, gp, seg, sp, o, p, PRE ? sl + B : nullptr);
                 i = 2 * B;
             }
-        } else {
-            round_batch<1, true, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, 0, gp, seg, sp, o, p, sl);
-            i = 1;
         }
         for (; i + B <= K; i += B)
-            round_batch<B, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
-        for (; i < K; ++i)
-            round_batch<1, false, BF16, MOM, WD, SPARSE, FROM_W>(acc, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
+            round_batch<B, BF16, MOM, WD, SPARSE, FROM_W>(acc, false, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
+        round_rest<B / 2, BF16, MOM, WD, SPARSE, FROM_W>(acc, i, K, wv, m, stride, gp, seg, sp, o, p);
         // ---- merge
         f8 dnew, wn;
 #pragma unroll

@@ -306,17 +306,51 @@ int enqueue_pipelined_merge(int flags)
 }
 
 // Work that an earlier call held back (HPSGD_OPT_FUSE) and that nothing has absorbed: a merge
-// (fuse 1) runs on its own, a batched local step (fuse 2) runs as an ordinary local step.
+// (fuse 1) runs on its own, local steps (fuse 2) run as ordinary local steps.
 int flush_deferred()
 {
     if (g.merge_deferred) {
         g.merge_deferred = false;
         TRY(enqueue_merge(g.deferred_flags));
     }
-    if (g.step_deferred) {
-        g.step_deferred = false;
-        TRY(enqueue_local(0, g.K, g.deferred_gp, g.deferred_sparse));
+    if (g.steps_held) {
+        // every maximal run of consecutive workers with a held step is one batched launch
+        const BatchPtrs all = g.deferred_gp;
+        const std::vector<char> held = g.step_held;
+        g.steps_held = 0;
+        std::fill(g.step_held.begin(), g.step_held.end(), 0);
+        for (int a = 0; a < g.K;) {
+            if (!held[a]) { ++a; continue; }
+            int b = a;
+            BatchPtrs gp{};
+            for (; b < g.K && held[b]; ++b) {
+                gp.dense[b - a] = all.dense[b];
+                gp.row_vals[b - a] = all.row_vals[b];
+                gp.slot[b - a] = all.slot[b];
+                gp.n_rows[b - a] = all.n_rows[b];
+            }
+            TRY(enqueue_local(a, b - a, gp, g.deferred_sparse));
+            a = b;
+        }
     }
+    return HPSGD_OK;
+}
+
+// Hold the local step of `worker` back (fuse 2).  A worker holds at most one step, and the held
+// steps are all dense or all sparse-row: anything else first launches what is held.
+int hold_step(int worker, const BatchPtrs& gp, int src, bool sparse)
+{
+    if (g.steps_held && (g.step_held[worker] || g.deferred_sparse != sparse)) TRY(flush_deferred());
+    if (!g.steps_held) {
+        g.deferred_gp = BatchPtrs{};
+        g.deferred_sparse = sparse;
+    }
+    g.deferred_gp.dense[worker] = gp.dense[src];
+    g.deferred_gp.row_vals[worker] = gp.row_vals[src];
+    g.deferred_gp.slot[worker] = gp.slot[src];
+    g.deferred_gp.n_rows[worker] = gp.n_rows[src];
+    g.step_held[worker] = 1;
+    ++g.steps_held;
     return HPSGD_OK;
 }
 
@@ -427,12 +461,13 @@ void launch_round_d(bool mom, bool wd, bool sparse, bool from_w, const FusedLaun
     else launch_round_s<BF16, false, false>(sparse, from_w, L);
 }
 
-// The deferred batched local step and the merge that follows it in one kernel per chunk (main
-// stream).  Afterwards every replica is a lazy clone of the new w.
+// The held-back local steps of all K workers and the merge that follows them in one kernel per
+// chunk (main stream).  Afterwards every replica is a lazy clone of the new w.
 int enqueue_round(int flags)
 {
     TRY(wait_pending_d2h(g.main));
-    g.step_deferred = false;
+    g.steps_held = 0;
+    std::fill(g.step_held.begin(), g.step_held.end(), 0);
     FusedLaunch L{};
     L.gp = g.deferred_gp;
     bool from_w = true;

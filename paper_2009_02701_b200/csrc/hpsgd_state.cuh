@@ -109,9 +109,10 @@ struct Ctx {
     bool reduce_outstanding = false;
     bool merge_deferred = false;           // fuse 1: hpsgd_sync_merge was called but its merge not yet enqueued
     int deferred_flags = 0;
-    bool step_deferred = false;            // fuse 2: a batched local step waits for the merge it will run with
-    BatchPtrs deferred_gp{};               //         its gradient pointers
-    bool deferred_sparse = false;
+    int steps_held = 0;                    // fuse 2: local steps held back for the merge they will run with
+    std::vector<char> step_held;           //         which workers have one (at most one each)
+    BatchPtrs deferred_gp{};               //         their gradient pointers, indexed by worker
+    bool deferred_sparse = false;          //         all of them sparse-row steps, or none
     std::vector<char> at_w;                // replica i equals w: no local step since its last clone
     std::vector<char> row_valid;           // row i of r holds replica i (else it is a lazy clone: read w)
     int64_t launches = 0;

@@ -540,6 +540,47 @@ def test_round_kernel_launches_one_kernel_per_round_and_writes_no_replica_row():
         assert bool(torch.isfinite(gu.dev_tensor(w, cfg.layout.P_pad)).all())
 
 
+def test_the_four_core_calls_alone_reach_the_round_kernel():
+    """hpsgd_init, hpsgd_local_step per worker, hpsgd_sync_merge, hpsgd_get_global with HPSGD_OPT_FUSE = 2:
+    K per-worker calls and the merge that follows are one launch; a worker that steps twice, or a merge
+    that finds only some workers stepped, falls back to separate launches.  Results as the oracle's."""
+    cfg = small("four_calls", 8, [30_000, 77], T=6, momentum=0.9, wd=1e-4)
+    o = gu.oracle_for(cfg)
+    with gu.session(cfg, fuse=2):
+        keep = []
+        hp.hpsgd_set_option(hp.HPSGD_OPT_PROFILE, 1)
+        for t in range(cfg.T):
+            before = hp.hpsgd_launch_count()
+            order = list(range(cfg.K)) if t % 2 == 0 else list(reversed(range(cfg.K)))   # any order of workers
+            if t == 3:
+                order.remove(5)                          # worker 5 sits this round out
+            for i in order:
+                inp = gu.host_inputs(cfg, i, t)
+                gu.gpu_step(cfg, i, inp, keep)
+                o.local_step(i, inp["flat"])
+            if t == 4:                                   # worker 2 steps a second time before the merge
+                inp = gu.host_inputs(cfg, 2, 100 + t)
+                gu.gpu_step(cfg, 2, inp, keep)
+                o.local_step(2, inp["flat"])
+            hp.hpsgd_sync_merge()
+            o.sync_merge()
+            launched = hp.hpsgd_launch_count() - before
+            if t == 3:
+                assert launched == 3                     # workers 0-4, workers 6-7, the merge
+            elif t == 4:
+                assert launched == 3                     # all eight, worker 2 again, the merge
+            else:
+                assert launched == 1
+        assert hp.hpsgd_profile_read(hp.HPSGD_KERNEL_ROUND)[1] == cfg.T - 2
+        w, D, rs, ms = gu.gpu_state(cfg)
+        gu.assert_bitwise(w, o.get_global(), "global model")
+        gu.assert_bitwise(D, o.get_pending(), "pending change")
+        for i in range(cfg.K):
+            gu.assert_bitwise(rs[i], o.get_replica(i), "replica %d" % i)
+            gu.assert_bitwise(ms[i], o.get_momentum(i), "momentum %d" % i)
+    o.close()
+
+
 def test_lazy_clones_under_every_other_call():
     """Interleave whole-round kernels with per-worker steps, idle workers, merges on their own,
     inspection and a change of schedule: replicas that exist only as 'w' must behave like rows."""
