@@ -65,16 +65,16 @@ def fused_bytes_per_index(cfg):
 # the indices of that launch), keyed by (kernel, K, gradient dtype), with the SHA-1 of the kernel source the
 # capture was taken from.  A changed source voids them.
 NCU_TRAFFIC = {
-    # profiles/round_kernel_cfg4_cut16M.txt: 2.176033 GB read + 1.103467 GB written over 16,000,000 indices
-    ('round_kernel', 16, 'f32'): {"bytes_per_index": 3.279500e9 / 16e6, "source_sha1": "8afef5adf5ca4ae72a3a02445d0d547a236f0fb7"},
-    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200026 GB read + 2.121719 GB written over 16,000,000 indices
-    ('merge_step_kernel', 16, 'f32'): {"bytes_per_index": 5.321745e9 / 16e6, "source_sha1": "8afef5adf5ca4ae72a3a02445d0d547a236f0fb7"},
-    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152243 GB read + 1.093507 GB written over 16,000,000 indices
-    ('merge_kernel', 16, 'f32'): {"bytes_per_index": 2.245750e9 / 16e6, "source_sha1": "8afef5adf5ca4ae72a3a02445d0d547a236f0fb7"},
-    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072010 GB read + 1.992945 GB written over 16,000,000 indices
-    ('local_step_kernel', 16, 'f32'): {"bytes_per_index": 5.064955e9 / 16e6, "source_sha1": "8afef5adf5ca4ae72a3a02445d0d547a236f0fb7"},
-    # profiles/round_kernel_cfg3.txt: 1.843403 GB read + 0.974397 GB written over 25,600,000 indices (weight decay)
-    ('round_kernel', 8, 'f32'): {"bytes_per_index": 2.817800e9 / 25.6e6, "source_sha1": "8afef5adf5ca4ae72a3a02445d0d547a236f0fb7"},
+    # profiles/round_kernel_cfg4_cut16M.txt: 2.176061 GB read + 1.104045 GB written over 16,000,000 indices
+    ('round_kernel', 16, 'f32'): {"bytes_per_index": 3.280106e9 / 16e6, "source_sha1": "2f17a8d97739018493e13686c185c65b2fcc6297"},
+    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200028 GB read + 2.122002 GB written over 16,000,000 indices
+    ('merge_step_kernel', 16, 'f32'): {"bytes_per_index": 5.322030e9 / 16e6, "source_sha1": "2f17a8d97739018493e13686c185c65b2fcc6297"},
+    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152078 GB read + 1.094110 GB written over 16,000,000 indices
+    ('merge_kernel', 16, 'f32'): {"bytes_per_index": 2.246188e9 / 16e6, "source_sha1": "2f17a8d97739018493e13686c185c65b2fcc6297"},
+    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072012 GB read + 1.992156 GB written over 16,000,000 indices
+    ('local_step_kernel', 16, 'f32'): {"bytes_per_index": 5.064168e9 / 16e6, "source_sha1": "2f17a8d97739018493e13686c185c65b2fcc6297"},
+    # profiles/round_kernel_cfg3.txt: 1.843402 GB read + 0.974462 GB written over 25,600,000 indices
+    ('round_kernel', 8, 'f32'): {"bytes_per_index": 2.817864e9 / 25.6e6, "source_sha1": "2f17a8d97739018493e13686c185c65b2fcc6297"},
 }
 
 
