@@ -311,11 +311,41 @@ def ulp_distance(a, b):
     return np.abs(a - b)
 
 
+PROBE_MIXES = ((16, 0), (16, 4), (12, 4), (13, 7), (12, 8), (8, 8), (4, 16), (0, 16))
+
+
+def do_nothing_rates(hp, torch, dev, row_bytes=256 << 20, iters=10):
+    """GB/s of a kernel with the hot kernels' access shape and no arithmetic, for each built mix of
+    read and write streams (hpsgd_probe_hbm): 20 arrays of 256 MB, far beyond the L2."""
+    buf = torch.empty(20 * row_bytes + 4096, dtype=torch.uint8, device=dev)
+    base = buf.data_ptr() + (-buf.data_ptr()) % 4096
+    torch.cuda.synchronize(dev)
+    hp.hpsgd_probe_hbm(base, 20 * row_bytes, 8, 8, row_bytes, 100)     # ~60 ms of load first: the clocks have dropped while the oracle ran
+    out = []
+    for n_read, n_write in PROBE_MIXES:
+        rate = max(hp.hpsgd_probe_hbm(base, 20 * row_bytes, n_read, n_write, row_bytes, iters) for _ in range(2))
+        out.append({"reads": n_read, "writes": n_write, "write_share": n_write / (n_read + n_write), "GB/s": rate})
+    del buf
+    torch.cuda.empty_cache()
+    return out
+
+
+def against_do_nothing(rates, share, achieved):
+    """The probe rate at the kernel's share of writes (linear between the two nearest built mixes)."""
+    pts = sorted((r["write_share"], r["GB/s"]) for r in rates)
+    rate = pts[-1][1]
+    for (s0, r0), (s1, r1) in zip(pts, pts[1:]):
+        if s0 <= share <= s1:
+            rate = r0 + (r1 - r0) * (share - s0) / (s1 - s0)
+            break
+    return {"write_share": share, "do_nothing_GB/s": rate, "kernel_over_do_nothing": achieved / rate}
+
+
 class GpuWorkload:
     """One workload resident on one GPU: arena and streams from torch, `nbuf` rounds of
     device-generated gradients, and the schedules of the path timed on them."""
 
-    KERNELS = ("local_step_kernel", "merge_kernel", "merge_step_kernel", "round_kernel")
+    KERNELS = ("local_step_kernel", "merge_kernel", "merge_step_kernel", "round_kernel", "merge_staged_kernel")
 
     def __init__(self, hp, torch, dev, cfg, args):
         self.hp, self.torch, self.dev, self.cfg, self.args = hp, torch, dev, cfg, args
@@ -332,7 +362,7 @@ class GpuWorkload:
         self.arena = torch.empty(self.nbytes + 256, dtype=torch.uint8, device=dev)
         self.base = self.arena.data_ptr() + (-self.arena.data_ptr()) % 256
         self.main, self.side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-        self.setup(args.pipeline, args.fuse, args.chunks)
+        self.setup(args.pipeline, args.fuse, args.chunks, args.staging)
         # inputs: `nbuf` rounds of gradients for all K workers, generated on the device
         self.nbuf = nbuf = args.grad_buffers
         self.row = -(-P_pad // 2048) * 2048          # every worker's gradient starts on a 4 KB boundary
@@ -355,7 +385,7 @@ class GpuWorkload:
                 hp.hpsgd_gen_grads(self.grads[b, i], i, b, self.kind, cfg.grad_scale)
         hp.hpsgd_synchronize()
 
-    def setup(self, pipeline, fuse, chunks):
+    def setup(self, pipeline, fuse, chunks, staging=0):
         hp, cfg = self.hp, self.cfg
         hp.hpsgd_destroy()
         if len(cfg.sizes) > 1:
@@ -370,6 +400,7 @@ class GpuWorkload:
         hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, self.args.overlap)
         hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, 1 if pipeline else chunks)
         hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
+        hp.hpsgd_set_option(hp.HPSGD_OPT_STAGING, staging)
         if cfg.sparse:
             hp.hpsgd_set_sparse_segment(*cfg.sparse)
         self.pipeline, self.fuse, self.chunks = pipeline, (0 if pipeline else fuse), (1 if pipeline else chunks)
@@ -456,6 +487,7 @@ class GpuWorkload:
             grad_bytes += active * 4 - (K * rows_total - active) * cols * self.gsz
         state_bytes = K * P * (8 + (8 if cfg.momentum else 0))        # r (and m) read and written
         return {"local_step_kernel": grad_bytes + state_bytes,
+                "merge_staged_kernel": merge_bytes_per_index(cfg) * P,
                 # pipelined: commit (w, D in; w out) + reduce (K r + w in; D out), two launches per merge
                 "merge_kernel": (12 + (K + 2) * 4) * P if self.pipeline else
                                 ((K + 4) * 4 * P if self.fuse == 2 else merge_bytes_per_index(cfg) * P),
@@ -463,6 +495,18 @@ class GpuWorkload:
                 # whole round in one kernel, one step per worker and period: no replica row is read
                 # or written; w, D, K m, K g in and w, D, K m out
                 "round_kernel": 16 * P + grad_bytes + (K * P * 8 if cfg.momentum else 0)}
+
+    def write_share(self, kernel):
+        """Share of the bytes a launch of `kernel` moves that are writes (HBM's rate depends on it)."""
+        cfg, K, P = self.cfg, self.cfg.K, self.cfg.P
+        mom = 4 if cfg.momentum else 0
+        written = {"local_step_kernel": K * P * (4 + mom),
+                   # pipelined: the commit writes w, the reduce writes D (two launches, one figure)
+                   "merge_kernel": (8 * P if (self.pipeline or self.fuse == 2) else (K + 2) * 4 * P),
+                   "merge_staged_kernel": (K + 2) * 4 * P,
+                   "merge_step_kernel": 8 * P + K * P * (4 + mom),
+                   "round_kernel": 8 * P + K * P * mom}[kernel]
+        return written / self.bytes_per_round()[kernel]
 
     def kernel_table(self, prof, peak):
         per_round = self.bytes_per_round()
@@ -486,7 +530,7 @@ class GpuWorkload:
         from oracle.ref import RefHPSGD
         hp, torch, cfg = self.hp, self.torch, self.cfg
         lay = cfg.layout
-        self.setup(self.pipeline, self.fuse if not self.pipeline else 0, self.chunks)
+        self.setup(self.pipeline, self.fuse if not self.pipeline else 0, self.chunks, self.args.staging)
         for t in range(cfg.T):
             self.regenerate(0, t)         # every round its own gradients, as in a real run (untimed)
             self.one_round(0)
@@ -537,7 +581,7 @@ class GpuWorkload:
         self.torch.cuda.empty_cache()
 
 
-def other_workload_entry(hp, torch, dev, name, args, peak):
+def other_workload_entry(hp, torch, dev, name, args, peak, rates=None):
     """A short timed run of another of the five workloads in the schedule being timed, with its
     parity figures (the oracle runs after the timed region)."""
     cfg = workloads.get(name)
@@ -551,6 +595,8 @@ def other_workload_entry(hp, torch, dev, name, args, peak):
              "gpu_launches": int(launches), "kernel": dominant, "kernel_avg_ms": kernels[dominant]["avg_ms"],
              "bytes_per_launch": kernels[dominant]["bytes_per_launch"], "achieved": kernels[dominant]["achieved"],
              "frac": kernels[dominant]["frac"], "frac_of_nominal_8TBs": kernels[dominant]["frac_of_nominal_8TBs"]}
+    if rates:
+        entry.update(against_do_nothing(rates, run.write_share(dominant), kernels[dominant]["achieved"]))
     state_mb = run.nbytes / 1e6
     if state_mb + run.grads.numel() * run.gsz / 1e6 < 126:
         entry["note"] = "L2-resident (state + gradients below the 126 MB L2) and launch-bound: GB/s here is not an HBM figure"
@@ -565,7 +611,7 @@ def other_workload_entry(hp, torch, dev, name, args, peak):
             "kernels": {k: {"launches": v["launches"], "avg_ms": v["avg_ms"], "bytes_per_launch": v["bytes_per_launch"],
                             "achieved": v["achieved"], "frac": v["frac"], "frac_of_nominal_8TBs": v["frac_of_nominal_8TBs"]}
                         for k, v in run.kernel_table(prof0, peak).items()}}
-        run.setup(args.pipeline, args.fuse, args.chunks)
+        run.setup(args.pipeline, args.fuse, args.chunks, args.staging)
     if args.parity:
         entry["parity"] = run.parity()
     run.release()
@@ -626,13 +672,15 @@ def run_gpu(args, cfg):
     # ---- the other schedules of the same path, timed briefly the same way (same inputs, same work)
     other = {}
     if args.other_schedule_steps > 0 and not args.per_worker:
-        for name, pipe, fuse in (("separate merge and local-step kernels on two streams", 0, 0),
-                                 ("pipelined commit + reduce on double-buffered replicas", 1, 0),
-                                 ("merge fused into the next local step", 0, 1),
-                                 ("one kernel per round (local steps + merge), replicas never stored", 0, 2)):
-            if (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
+        for name, pipe, fuse, staging in (
+                ("separate merge and local-step kernels on two streams", 0, 0, 0),
+                ("separate kernels, the merge's tiles staged through shared memory by bulk-async copies", 0, 0, 1),
+                ("pipelined commit + reduce on double-buffered replicas", 1, 0, 0),
+                ("merge fused into the next local step", 0, 1, 0),
+                ("one kernel per round (local steps + merge), replicas never stored", 0, 2, 0)):
+            if not staging and (pipe, fuse if not pipe else 0) == (args.pipeline, 0 if args.pipeline else args.fuse):
                 continue
-            run.setup(pipe, fuse, 1)
+            run.setup(pipe, fuse, 1, staging)
             ms, n_launch, prof_o = run.timed(args.other_schedule_steps, 3)
             ms /= args.other_schedule_steps
             other[name] = {"ms_per_step": ms, "value": K * P / (ms * 1e-3), "steps": args.other_schedule_steps,
@@ -640,7 +688,7 @@ def run_gpu(args, cfg):
                            "kernels": {k: {"launches": v["launches"], "avg_ms": v["avg_ms"], "achieved": v["achieved"],
                                            "frac_of_nominal_8TBs": v["frac_of_nominal_8TBs"]}
                                        for k, v in run.kernel_table(prof_o, peak).items()}}
-        run.setup(args.pipeline, args.fuse, args.chunks)
+        run.setup(args.pipeline, args.fuse, args.chunks, args.staging)
 
     # ---- end to end: host gradient buffers in, host copy of the global model out, every step
     e2e = None
@@ -650,13 +698,21 @@ def run_gpu(args, cfg):
     line = None
     if rank == 0:
         parity = run.parity() if args.parity else None
+        share = run.write_share(dominant)
         run.release()
+        rates = None
+        if args.probe:
+            rates = do_nothing_rates(hp, torch, dev)
+            roofline["do_nothing"] = {
+                "method": "hpsgd_probe_hbm: R read + W write arrays of 256 MB, one block per 128 groups of 8 floats, "
+                          "256-bit accesses, sums only; best of two runs of 10 timed launches each, CUDA events",
+                "rates": rates, **against_do_nothing(rates, share, kernels[dominant]["achieved"])}
         # ---- the other four workloads, briefly, each with its parity figures
         others = {}
         if args.other_workload_steps > 0 and not args.max_params:
             for name in workloads.names():
                 if name != cfg.name:
-                    others[name] = other_workload_entry(hp, torch, dev, name, args, peak)
+                    others[name] = other_workload_entry(hp, torch, dev, name, args, peak, rates)
         cpu = None
         if args.cpu_seconds > 0:
             eps, rounds, spent, desc, _ = oracle_sample_run(cfg, args.cpu_seconds)
@@ -672,7 +728,7 @@ def run_gpu(args, cfg):
                              "fuse": 0 if args.pipeline else args.fuse,
                              "fuse_meaning": "2: one kernel per round (batched local step inside the kernel of the merge "
                                              "that follows it); 1: merge carried into the next local step; 0: separate kernels",
-                             "pipelined_commit_reduce": args.pipeline,
+                             "pipelined_commit_reduce": args.pipeline, "staged_merge": args.staging,
                              "local_step_call": "per worker" if args.per_worker else "all K in one call"},
                 "l2": "inputs larger than L2 (state + gradients are tens of GB)",
                 "multi_gpu": "independent replicas, no inter-GPU exchange"}),
@@ -762,6 +818,10 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU oracle baseline budget (0 = skip)")
     ap.add_argument("--other-workload-steps", type=int, default=10,
                     help="timed rounds for each of the other four workloads, reported under `workloads` (0 = skip)")
+    ap.add_argument("--staging", type=int, default=0,
+                    help="1: the stand-alone merge (fuse 0 or 1) stages its tiles through shared memory with bulk-async copies")
+    ap.add_argument("--probe", type=int, default=1,
+                    help="1: also measure what HBM gives a do-nothing kernel for each read/write mix (hpsgd_probe_hbm)")
     ap.add_argument("--parity", type=int, default=1,
                     help="1: after the timed regions, run each workload's T rounds and compare a sample with the CPU oracle")
     ap.add_argument("--max-params", type=int, default=0,

@@ -41,7 +41,7 @@ typedef enum hpsgd_status {
     HPSGD_E_STATE = -2,       /* call not legal in the current state (e.g. before hpsgd_init) */
     HPSGD_E_NOMEM = -3,       /* arena too small or device allocation failed */
     HPSGD_E_CUDA = -4,        /* a CUDA call failed; see hpsgd_last_error() */
-    HPSGD_E_TIMEOUT = -5,     /* reserved: no kernel of this library waits on the device, so nothing returns it */
+    HPSGD_E_TIMEOUT = -5,     /* a bounded device-side wait ran out (only the staged merge of HPSGD_OPT_STAGING has one) */
     HPSGD_E_UNSUPPORTED = -6  /* size beyond a documented limit */
 } hpsgd_status;
 
@@ -85,6 +85,18 @@ enum {
                                    For callers whose gradients are already resident (a simulation, a
                                    benchmark) 2 is the fastest; a trainer that computes the next gradients
                                    while the merge runs wants 0. */
+    HPSGD_OPT_STAGING = 9,      /* 0 (default): the merge reads and writes global memory directly, one 256-bit
+                                   access per thread and array.  1: the stand-alone merge kernel (HPSGD_OPT_FUSE
+                                   0 or 1, replica-change form, K <= 32) instead brings the K + 2 tiles of a block
+                                   into shared memory with bulk asynchronous copies that complete on an mbarrier,
+                                   and writes its K + 2 result tiles back with bulk stores.  Same operations in
+                                   the same order: bit-identical.  It exists so that the two ways of issuing the
+                                   memory traffic can be timed against each other on the same state; the merge has
+                                   no data reuse for shared memory to exploit, and the plain form is as fast or
+                                   faster.  The staged kernel is the only device code of this library that waits
+                                   (on its own loads, a bounded number of tries): if a wait ever runs out, the
+                                   block writes nothing and the next call that waits for the device returns
+                                   HPSGD_E_TIMEOUT. */
     HPSGD_OPT_DEBUG_GROUP_LIMIT = 8 /* Checked build (compiled with -DHPSGD_DEBUG) only; HPSGD_E_UNSUPPORTED
                                    otherwise.  In that build every hot kernel tests each 8-element group
                                    index against the number of groups of a flat buffer before touching
@@ -97,7 +109,8 @@ enum {
 
 /* Kernel kinds of hpsgd_profile_read. */
 enum { HPSGD_KERNEL_LOCAL_STEP = 0, HPSGD_KERNEL_MERGE = 1, HPSGD_KERNEL_MERGE_STEP = 2 /* fuse 1 */,
-       HPSGD_KERNEL_ROUND = 3 /* fuse 2: local steps + merge */ };
+       HPSGD_KERNEL_ROUND = 3 /* fuse 2: local steps + merge */,
+       HPSGD_KERNEL_MERGE_STAGED = 4 /* the merge under HPSGD_OPT_STAGING */ };
 
 enum { HPSGD_F32 = 0, HPSGD_BF16 = 1 };
 
@@ -416,12 +429,29 @@ int hpsgd_synchronize(void);
 
 /*
  * With HPSGD_OPT_PROFILE on: total device milliseconds and number of launches of one kind
- * of kernel (HPSGD_KERNEL_*: local step, merge, merge + next local step, whole round) since the last
+ * of kernel (HPSGD_KERNEL_*: local step, merge, merge + next local step, whole round, staged merge) since the last
  * read of that kind, measured with CUDA event pairs recorded around each launch on the
  * stream it ran on.  Launches any deferred merge, synchronises, and resets that kind's
  * totals.  Any out pointer may be NULL.
  */
 int hpsgd_profile_read(int kind, double* ms, int64_t* launches);
+
+/*
+ * What HBM gives a kernel that reads n_read arrays and writes n_write arrays per index with the
+ * access shape of this library's hot kernels (one block per 128 groups of 8 floats, 256-bit
+ * loads and stores, all loads requested before the first use) and next to no arithmetic: the
+ * ceiling a hot kernel with that share of writes is to be compared with (DRAM loses bandwidth
+ * to read/write turnarounds, so the ceiling depends on the mix).  (The paper has no counterpart;
+ * this is a measuring aid.)  `scratch` is device memory lent for the duration of the call
+ * (4096-byte aligned, at least (n_read + n_write) * row_bytes; it is overwritten with zeros);
+ * row_bytes is the length of each array (a multiple of 4096; use arrays that together exceed the
+ * L2 cache several times).  Runs two untimed and `iters` timed launches on a stream of its own,
+ * waits, and returns (n_read + n_write) * row_bytes * iters / time in *gb_per_s (1e9 bytes/s).
+ * Built mixes (n_read, n_write): (16,0) (12,4) (16,4) (13,7) (12,8) (8,8) (4,16) (0,16); others
+ * give HPSGD_E_UNSUPPORTED.  Needs no hpsgd_init and touches no state of the library.  Blocking.
+ */
+int hpsgd_probe_hbm(void* scratch, size_t scratch_bytes, int n_read, int n_write, int64_t row_bytes, int iters,
+                    double* gb_per_s);
 
 /* Enqueue what HPSGD_OPT_FUSE held back (a merge, or a batched local step), if anything (does not wait). */
 int hpsgd_flush(void);

@@ -17,7 +17,9 @@ HPSGD_E_CUDA, HPSGD_E_TIMEOUT, HPSGD_E_UNSUPPORTED = -4, -5, -6
 HPSGD_OPT_WEIGHT_DECAY, HPSGD_OPT_STALENESS, HPSGD_OPT_GRAD_DTYPE = 1, 2, 3
 HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE, HPSGD_OPT_FUSE = 4, 5, 6, 7
 HPSGD_OPT_DEBUG_GROUP_LIMIT = 8
+HPSGD_OPT_STAGING = 9
 HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP, HPSGD_KERNEL_ROUND = 0, 1, 2, 3
+HPSGD_KERNEL_MERGE_STAGED = 4
 HPSGD_F32, HPSGD_BF16 = 0, 1
 HPSGD_GEN_UNIFORM, HPSGD_GEN_GAUSS = 0, 1
 HPSGD_ARENA_MOMENTUM = 1
@@ -76,6 +78,7 @@ SIGNATURES = {
     "hpsgd_gen_row_vals": (_ci, [_vp, _ci, _ci, _ci, _f64, _vp, ctypes.c_int32]),
     "hpsgd_synchronize": (_ci, []),
     "hpsgd_profile_read": (_ci, [_ci, _P(_f64), _P(_i64)]),
+    "hpsgd_probe_hbm": (_ci, [_vp, _sz, _ci, _ci, _i64, _ci, _P(_f64)]),
     "hpsgd_flush": (_ci, []),
     "hpsgd_launch_count": (_i64, []),
     "hpsgd_last_error": (ctypes.c_char_p, []),
@@ -307,6 +310,14 @@ def hpsgd_profile_read(kind):
     ms, n = _f64(), _i64()
     _check(load().hpsgd_profile_read(int(kind), ctypes.byref(ms), ctypes.byref(n)))
     return ms.value, n.value
+
+
+def hpsgd_probe_hbm(scratch, scratch_bytes, n_read, n_write, row_bytes, iters):
+    """GB/s (1e9 bytes/s) of a kernel that only reads n_read and writes n_write arrays of row_bytes."""
+    out = _f64()
+    _check(load().hpsgd_probe_hbm(_ptr(scratch), int(scratch_bytes), int(n_read), int(n_write), int(row_bytes),
+                                  int(iters), ctypes.byref(out)))
+    return out.value
 
 
 def hpsgd_flush():

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhpsgd.so")
 SOURCES = [os.path.join(CSRC, "hpsgd_api.cu")]
 DEPENDS = SOURCES + [os.path.join(CSRC, "hpsgd_kernels.cuh"), os.path.join(CSRC, "hpsgd_state.cuh"),
-                     os.path.join(CSRC, "hpsgd_schedule.cuh"),
+                     os.path.join(CSRC, "hpsgd_schedule.cuh"), os.path.join(CSRC, "hpsgd_staged.cuh"),
                      os.path.join(os.path.dirname(HERE), "include", "hpsgd.h")]
 # --fmad=false: the compiler never contracts a*b+c on its own; fused multiply-adds are
 # written explicitly where the update rule has them.

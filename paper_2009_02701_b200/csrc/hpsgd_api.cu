@@ -259,6 +259,10 @@ int hpsgd_set_option(int key, double value)
         g.fuse = (int)value;
         if (!lazy_clones() && !g.pipeline) TRY(materialize_clones());   // the other schedules read replica rows
         return HPSGD_OK;
+    case HPSGD_OPT_STAGING:
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "staging must be 0 or 1");
+        g.staging = (int)value;
+        return HPSGD_OK;
     case HPSGD_OPT_DEBUG_GROUP_LIMIT:
 #ifdef HPSGD_DEBUG
         if (!(value >= -1.0 && value <= (double)(g.P_pad / 8) && value == (double)(int64_t)value))
@@ -732,7 +736,7 @@ int hpsgd_gen_row_vals(void* out, int worker, int step, int kind, double scale,
 int hpsgd_profile_read(int kind, double* ms, int64_t* launches)
 {
     TRY(need_init());
-    if (kind < 0 || kind > 3) return fail(HPSGD_E_BADARG, "unknown kernel kind %d", kind);
+    if (kind < 0 || kind > 4) return fail(HPSGD_E_BADARG, "unknown kernel kind %d", kind);
     TRY(flush_deferred());
     TRY(sync_all());
     TRY(prof_resolve());
@@ -744,6 +748,88 @@ int hpsgd_profile_read(int kind, double* ms, int64_t* launches)
 }
 
 int64_t hpsgd_launch_count(void) { return g.inited ? g.launches : 0; }
+
+// ------------------------------------------------------------------------- bandwidth probe
+}  // extern "C"
+
+namespace {
+
+template <int R, int W>
+void launch_probe(cudaStream_t s, float* base, int64_t row_floats, int64_t n_groups)
+{
+    // the W destination rows follow the R source rows; with nothing to write the (never taken) store aims at row 0
+    float* dst = W > 0 ? base + (int64_t)R * row_floats : base;
+    stream_probe_kernel<R, W><<<hot_grid(n_groups), kHotThreads, 0, s>>>(base, dst, row_floats, n_groups);
+}
+
+// The read / write mixes the probe is built for: (16, 0) pure reads ... (0, 16) pure writes.
+bool probe_dispatch(int R, int W, cudaStream_t s, float* base, int64_t row_floats, int64_t n_groups)
+{
+#define HPSGD_PROBE_CASE(r, w) if (R == r && W == w) { launch_probe<r, w>(s, base, row_floats, n_groups); return true; }
+    HPSGD_PROBE_CASE(16, 0)
+    HPSGD_PROBE_CASE(12, 4)
+    HPSGD_PROBE_CASE(16, 4)
+    HPSGD_PROBE_CASE(13, 7)
+    HPSGD_PROBE_CASE(12, 8)
+    HPSGD_PROBE_CASE(8, 8)
+    HPSGD_PROBE_CASE(4, 16)
+    HPSGD_PROBE_CASE(0, 16)
+#undef HPSGD_PROBE_CASE
+    return false;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hpsgd_probe_hbm(void* scratch, size_t scratch_bytes, int n_read, int n_write, int64_t row_bytes, int iters,
+                    double* gb_per_s)
+{
+    if (!scratch || reinterpret_cast<uintptr_t>(scratch) % kPageBytes)
+        return fail(HPSGD_E_BADARG, "scratch must be a 4096-byte aligned device pointer");
+    if (row_bytes <= 0 || row_bytes % (int64_t)kPageBytes) return fail(HPSGD_E_BADARG, "row_bytes must be a positive multiple of 4096");
+    if (n_read < 0 || n_write < 0 || n_read + n_write <= 0) return fail(HPSGD_E_BADARG, "need at least one stream");
+    if (iters <= 0 || iters > 10000) return fail(HPSGD_E_BADARG, "iters must be in [1, 10000]");
+    if (!gb_per_s) return fail(HPSGD_E_BADARG, "gb_per_s is NULL");
+    const int rows = n_read + n_write;
+    if (scratch_bytes / (size_t)row_bytes < (size_t)rows)
+        return fail(HPSGD_E_NOMEM, "scratch of %zu bytes is smaller than the %d rows of %lld bytes needed", scratch_bytes,
+                    rows, (long long)row_bytes);
+    cudaStream_t s = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    float* base = static_cast<float*>(scratch);
+    const int64_t row_floats = row_bytes / 4, n_groups = row_bytes / 32;
+    int rc = HPSGD_OK;
+    float ms = 0.f;
+    cudaError_t e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreate(&a);
+    if (e == cudaSuccess) e = cudaEventCreate(&b);
+    // zeros: sums stay finite however often the probe runs over the same memory
+    if (e == cudaSuccess) e = cudaMemsetAsync(scratch, 0, (size_t)rows * (size_t)row_bytes, s);
+    if (e == cudaSuccess) {
+        for (int it = -2; it < iters && rc == HPSGD_OK; ++it) {          // two untimed launches first
+            if (it == 0) e = cudaEventRecord(a, s);
+            if (e != cudaSuccess) break;
+            if (!probe_dispatch(n_read, n_write, s, base, row_floats, n_groups))
+                rc = fail(HPSGD_E_UNSUPPORTED, "no probe for %d read and %d write streams; built: (16,0) (12,4) (16,4) (13,7) "
+                                               "(12,8) (8,8) (4,16) (0,16)", n_read, n_write);
+        }
+    }
+    if (e == cudaSuccess && rc == HPSGD_OK) e = cudaEventRecord(b, s);
+    if (e == cudaSuccess && rc == HPSGD_OK) e = cudaEventSynchronize(b);
+    if (e == cudaSuccess && rc == HPSGD_OK) e = cudaEventElapsedTime(&ms, a, b);
+    if (e == cudaSuccess && rc == HPSGD_OK) e = cudaGetLastError();
+    if (s) { cudaStreamSynchronize(s); cudaStreamDestroy(s); }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (rc != HPSGD_OK) return rc;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HPSGD_E_CUDA, "bandwidth probe failed: %s", cudaGetErrorString(e));
+    }
+    *gb_per_s = (double)(n_read + n_write) * (double)row_bytes * iters / (ms * 1e-3) / 1e9;
+    return HPSGD_OK;
+}
 
 }  // extern "C"
 

@@ -191,6 +191,26 @@ void launch_merge(cudaStream_t s, int64_t o0, int64_t n, int flags)
     merge_kernel<KT><<<hot_grid(n), kHotThreads, 0, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags, group_limit());
 }
 
+// The same merge with its tiles staged through shared memory by bulk-async copies (HPSGD_OPT_STAGING).
+int launch_merge_staged(cudaStream_t s, int64_t o0, int64_t n, int flags)
+{
+    const size_t smem = (size_t)(g.K + 2) * kStageTileFloats * sizeof(float);
+    if (!g.staged_attr) {
+        CUDA_TRY(cudaFuncSetAttribute(merge_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)((kMaxBatch + 2) * kStageTileFloats * sizeof(float))));
+        g.staged_attr = true;
+    }
+    const int64_t tiles = (n + kStageGroups - 1) / kStageGroups;
+    merge_staged_kernel<<<(unsigned)tiles, kHotThreads, smem, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags, group_limit());
+    g.staged_ran = true;
+    return HPSGD_OK;
+}
+
+bool staged_merge()
+{
+    return g.staging && g.form == HPSGD_FORM_REPLICA_CHANGE && !g.pipeline && !lazy_clones() && g.K <= kMaxBatch;
+}
+
 template <int KT>
 void launch_merge_lazy(cudaStream_t s, const ReducePtrs& rp, int64_t o0, int64_t n, int flags)
 {
@@ -222,7 +242,7 @@ int enqueue_merge(int flags)
             g.local_recorded[c] = 0;
         }
         EventPair ep{};
-        TRY(prof_begin(s, HPSGD_KERNEL_MERGE, &ep));
+        TRY(prof_begin(s, (!lazy && staged_merge()) ? HPSGD_KERNEL_MERGE_STAGED : HPSGD_KERNEL_MERGE, &ep));
         if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) {
             switch (g.K) {
             case 4: launch_accum_merge<4>(s, lo, hi - lo, flags); break;
@@ -237,6 +257,8 @@ int enqueue_merge(int flags)
             case 16: launch_merge_lazy<16>(s, rp, lo, hi - lo, flags); break;
             default: launch_merge_lazy<0>(s, rp, lo, hi - lo, flags); break;
             }
+        } else if (staged_merge()) {
+            TRY(launch_merge_staged(s, lo, hi - lo, flags));
         } else {
             switch (g.K) {
             case 4: launch_merge<4>(s, lo, hi - lo, flags); break;

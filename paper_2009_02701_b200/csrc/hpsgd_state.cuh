@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "hpsgd_kernels.cuh"
+#include "hpsgd_staged.cuh"
 
 namespace {
 
@@ -100,6 +101,9 @@ struct Ctx {
     int64_t merges = 0;
     int form = HPSGD_FORM_REPLICA_CHANGE;  // what the workers carry: replica change or accumulated gradients
     int fuse = 0;                          // carry a merge into the next batched local step
+    int staging = 0;                       // merges bring their tiles through shared memory with bulk-async copies
+    bool staged_ran = false;               //   ... one has been launched since the last look at its time-out count
+    bool staged_attr = false;              //   ... its shared-memory size has been opted into on this device
     int pipeline = 0;                      // commit/reduce split on double-buffered replicas
     float* wbuf[2] = {nullptr, nullptr};   // pipeline: global model of the current / other period
     float* rbuf[2] = {nullptr, nullptr};   // pipeline: replica sets of the current / other period
@@ -124,8 +128,8 @@ struct Ctx {
     bool stage_used[2] = {false, false};
     int stage_next = 0;
     std::vector<EventPair> prof;           // profiling
-    double prof_ms[4] = {0, 0, 0, 0};
-    int64_t prof_launches[4] = {0, 0, 0, 0};
+    double prof_ms[5] = {0, 0, 0, 0, 0};
+    int64_t prof_launches[5] = {0, 0, 0, 0, 0};
     int64_t debug_limit = -1;              // checked build: groups per flat buffer the kernels test against (< 0: P_pad / 8)
 } g;
 
@@ -154,6 +158,23 @@ int debug_poll()
                     rep.kernel, what[rep.code < 4 ? rep.code : 0], rep.index, rep.limit);
     }
 #endif
+    return HPSGD_OK;
+}
+
+// The staged merge waits (bounded) for its own bulk loads; blocks whose wait ran out counted
+// themselves.  Called where the host has just waited for the device.
+int staged_poll()
+{
+    if (!g.staged_ran) return HPSGD_OK;
+    g.staged_ran = false;
+    unsigned int n = 0;
+    CUDA_TRY(cudaMemcpyFromSymbol(&n, g_stage_timeouts, sizeof n));
+    if (n != 0) {
+        const unsigned int zero = 0;
+        CUDA_TRY(cudaMemcpyToSymbol(g_stage_timeouts, &zero, sizeof zero));
+        return fail(HPSGD_E_TIMEOUT, "staged merge: %u blocks gave up waiting for their bulk loads and wrote nothing; "
+                                     "the state is no longer consistent", n);
+    }
     return HPSGD_OK;
 }
 
@@ -315,6 +336,7 @@ int sync_all()
     if (g.copy) CUDA_TRY(cudaStreamSynchronize(g.copy));
     if (g.d2h) CUDA_TRY(cudaStreamSynchronize(g.d2h));
     g.d2h_outstanding = false;
+    TRY(staged_poll());
     return debug_poll();
 }
 

@@ -41,7 +41,7 @@ def to_device(a: np.ndarray) -> torch.Tensor:
 
 @contextlib.contextmanager
 def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, pipeline=0, lend_arena=False, streams=False,
-            canary=False):
+            canary=False, staging=0):
     """hpsgd_init for a workload (layout, options, optional lent arena/streams); destroys on exit."""
     hp.hpsgd_destroy()
     lay = cfg.layout
@@ -76,6 +76,8 @@ def session(cfg, *, staleness=None, overlap=1, chunks=1, fuse=0, form=0, pipelin
         hp.hpsgd_set_option(hp.HPSGD_OPT_OVERLAP, overlap)
         hp.hpsgd_set_option(hp.HPSGD_OPT_CHUNKS, chunks)
         hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, fuse)
+        if staging:
+            hp.hpsgd_set_option(hp.HPSGD_OPT_STAGING, staging)
         if cfg.sparse:
             hp.hpsgd_set_sparse_segment(*cfg.sparse)
         yield keep

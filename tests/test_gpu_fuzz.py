@@ -124,3 +124,54 @@ def test_random_call_sequences_gradient_accumulation_form(seed):
                 look("seed %d after op %d" % (seed, op_no))
         look("seed %d at the end" % seed)
     o.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_call_sequences_sparse_rows(seed):
+    """The same with a sparse-row tensor in the layout: batched and per-worker sparse-row steps mixed with
+    dense ones (which hold back, flush and share the per-worker row -> slot maps differently), fp32 and bf16."""
+    rng = np.random.default_rng(9000 + seed)
+    K = int(rng.choice([2, 3, 4, 8, 16]))
+    rows, cols = int(rng.integers(5, 200)), int(rng.choice([8, 16, 64]))
+    sizes = [int(rng.integers(1, 5000)), rows * cols, int(rng.integers(1, 5000))]
+    momentum = float(rng.choice([0.0, 0.9]))
+    wd = float(rng.choice([0.0, 1e-3]))
+    pipeline = int(rng.random() < 0.2)
+    cfg = Workload("fuzz_sparse", K=K, sizes=tuple(sizes), T=0, lr=0.05, momentum=momentum, weight_decay=wd,
+                   seed=300 + seed, grad_kind="gauss", grad_scale=1e-2, grad_dtype=str(rng.choice(["f32", "bf16"])),
+                   sparse=(1, rows, cols))
+    o = gu.oracle_for(cfg)
+    keep = []
+    step = 0
+    with gu.session(cfg, overlap=int(rng.choice([0, 1])), chunks=1 if pipeline else int(rng.choice([1, 3])),
+                    fuse=int(rng.choice([0, 1, 2])), pipeline=pipeline, lend_arena=bool(rng.random() < 0.5)):
+        for op_no in range(30):
+            op = rng.choice(["all_ex", "all_ex", "all_ex", "some_ex", "some_dense", "merge", "merge", "merge", "sync",
+                             "look", "fuse"])
+            if op == "all_ex":
+                descs = []
+                for i in range(K):
+                    inp = gu.host_inputs(cfg, i, step)
+                    g, idx, vals = gu.to_device(inp["padded"]), gu.to_device(inp["rows"]), gu.to_device(inp["vals"].reshape(-1))
+                    keep += [g, idx, vals]
+                    descs.append(hp.make_desc(g, idx, len(inp["rows"]), vals))
+                    gu.oracle_step(o, cfg, i, inp)
+                hp.hpsgd_local_step_all_ex(descs)
+                step += 1
+            elif op in ("some_ex", "some_dense"):
+                for i in rng.permutation(K)[:int(rng.integers(1, K + 1))]:
+                    inp = gu.host_inputs(cfg, int(i), step)
+                    gu.gpu_step(cfg, int(i), inp, keep, sparse_api=(op == "some_ex"))
+                    gu.oracle_step(o, cfg, int(i), inp, sparse_api=(op == "some_ex"))
+                step += 1
+            elif op == "merge":
+                hp.hpsgd_sync_merge()
+                o.sync_merge()
+            elif op == "sync":
+                hp.hpsgd_synchronize()
+            elif op == "look":
+                compare(cfg, o, "seed %d after op %d" % (seed, op_no))
+            elif op == "fuse" and not pipeline:
+                hp.hpsgd_set_option(hp.HPSGD_OPT_FUSE, int(rng.choice([0, 1, 2])))
+        compare(cfg, o, "seed %d at the end" % seed)
+    o.close()
