@@ -16,9 +16,9 @@
 // its own bulk loads complete on.  The wait is a bounded try_wait loop; a block whose wait runs
 // out counts itself in g_stage_timeouts, waits once more (bounded) so that no copy is still on
 // its way into shared memory that the next block will own, writes nothing and returns.  The
-// host turns a non-zero count into HPSGD_E_TIMEOUT at its next synchronisation.  No cluster
-// launch and no multicast anywhere: every copy is between this GPU's global memory and the
-// issuing block's own shared memory.
+// host turns a non-zero count into HPSGD_E_TIMEOUT at its next synchronisation.  Blocks are
+// launched without clusters and every copy is between this GPU's global memory and the issuing
+// block's own shared memory: nothing is delivered to another block.
 #pragma once
 
 #include "hpsgd_kernels.cuh"
@@ -38,7 +38,7 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  :: "r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
