@@ -43,7 +43,8 @@ def test_checked_build_gives_the_same_results(checked_library):
             gu.run_both(cfg, cfg.T, fuse=2, batched=True)
     cfg = small("chk_multi", 8, [70_001, 33, 4096], T=4, wd=5e-4)
     for kw in (dict(), dict(fuse=1, batched=True, chunks=3), dict(fuse=2, batched=True, chunks=2),
-               dict(pipeline=1, batched=True), dict(batched=True, chunks=5, overlap=0)):
+               dict(pipeline=1, batched=True), dict(batched=True, chunks=5, overlap=0),
+               dict(chunks=2, session_kw=dict(staging=1))):
         gu.run_both(cfg, cfg.T, **kw)
     for dtype in ("f32", "bf16"):
         cfg = small("chk_sparse", 5, [1000, 300 * 64, 777, 64], T=4, dtype=dtype, sparse=(1, 300, 64), scale=1e-3)
@@ -92,15 +93,15 @@ def test_checked_build_refuses_bad_row_lists_before_launching(checked_library):
     assert torch.equal(r, keep)
 
 
-@pytest.mark.parametrize("fuse,batched", [(0, False), (0, True), (1, True), (2, True)])
-def test_kernel_guard_records_and_skips(checked_library, fuse, batched):
+@pytest.mark.parametrize("fuse,batched,staging", [(0, False, 0), (0, True, 0), (1, True, 0), (2, True, 0), (0, True, 1)])
+def test_kernel_guard_records_and_skips(checked_library, fuse, batched, staging):
     """With the limit lowered to half the buffer the kernels skip the upper half (in-bounds memory
     that the guard now calls out of range), the next synchronisation reports it, and the state
     stays usable."""
     cfg = small("chk_guard", 4, [8192 * 8], T=1, momentum=0.9)
     groups = cfg.layout.P_pad // 8
     half = groups // 2
-    with gu.session(cfg, fuse=fuse):
+    with gu.session(cfg, fuse=fuse, staging=staging):
         inputs = [gu.host_inputs(cfg, i, 0) for i in range(cfg.K)]
         stacked = np.stack([inp["padded"] for inp in inputs])
         dev_g = gu.to_device(stacked.reshape(-1))
