@@ -314,25 +314,29 @@ def ulp_distance(a, b):
 PROBE_MIXES = ((16, 0), (16, 4), (12, 4), (13, 7), (12, 8), (8, 8), (4, 16), (0, 16))
 
 
-def do_nothing_rates(hp, torch, dev, row_bytes=256 << 20, iters=10):
+def do_nothing_rates(hp, torch, dev, cfg):
     """GB/s of a kernel with the hot kernels' access shape and no arithmetic, for each built mix of
-    read and write streams (hpsgd_probe_hbm): 20 arrays of 256 MB, far beyond the L2."""
+    read and write streams (hpsgd_probe_hbm), on arrays as long as one flat buffer of the workload
+    (at most 512 MB each), so that a short launch is compared with an equally short one."""
+    row_bytes = min(512 << 20, -(-cfg.layout.P_pad * 4 // 4096) * 4096)
+    iters = int(min(500, max(10, 4e9 // (16 * row_bytes))))
     buf = torch.empty(20 * row_bytes + 4096, dtype=torch.uint8, device=dev)
     base = buf.data_ptr() + (-buf.data_ptr()) % 4096
     torch.cuda.synchronize(dev)
-    hp.hpsgd_probe_hbm(base, 20 * row_bytes, 8, 8, row_bytes, 100)     # ~60 ms of load first: the clocks have dropped while the oracle ran
+    warm = int(min(10000, max(1, 4e10 // (16 * row_bytes))))
+    hp.hpsgd_probe_hbm(base, 20 * row_bytes, 8, 8, row_bytes, warm)    # ~60 ms of load first: the clocks drop while the oracle runs
     out = []
     for n_read, n_write in PROBE_MIXES:
         rate = max(hp.hpsgd_probe_hbm(base, 20 * row_bytes, n_read, n_write, row_bytes, iters) for _ in range(2))
         out.append({"reads": n_read, "writes": n_write, "write_share": n_write / (n_read + n_write), "GB/s": rate})
     del buf
     torch.cuda.empty_cache()
-    return out
+    return {"array_bytes": row_bytes, "launches_timed": iters, "rates": out}
 
 
 def against_do_nothing(rates, share, achieved):
     """The probe rate at the kernel's share of writes (linear between the two nearest built mixes)."""
-    pts = sorted((r["write_share"], r["GB/s"]) for r in rates)
+    pts = sorted((r["write_share"], r["GB/s"]) for r in rates["rates"])
     rate = pts[-1][1]
     for (s0, r0), (s1, r1) in zip(pts, pts[1:]):
         if s0 <= share <= s1:
@@ -581,7 +585,7 @@ class GpuWorkload:
         self.torch.cuda.empty_cache()
 
 
-def other_workload_entry(hp, torch, dev, name, args, peak, rates=None):
+def other_workload_entry(hp, torch, dev, name, args, peak):
     """A short timed run of another of the five workloads in the schedule being timed, with its
     parity figures (the oracle runs after the timed region)."""
     cfg = workloads.get(name)
@@ -595,8 +599,7 @@ def other_workload_entry(hp, torch, dev, name, args, peak, rates=None):
              "gpu_launches": int(launches), "kernel": dominant, "kernel_avg_ms": kernels[dominant]["avg_ms"],
              "bytes_per_launch": kernels[dominant]["bytes_per_launch"], "achieved": kernels[dominant]["achieved"],
              "frac": kernels[dominant]["frac"], "frac_of_nominal_8TBs": kernels[dominant]["frac_of_nominal_8TBs"]}
-    if rates:
-        entry.update(against_do_nothing(rates, run.write_share(dominant), kernels[dominant]["achieved"]))
+    share = run.write_share(dominant)
     state_mb = run.nbytes / 1e6
     if state_mb + run.grads.numel() * run.gsz / 1e6 < 126:
         entry["note"] = "L2-resident (state + gradients below the 126 MB L2) and launch-bound: GB/s here is not an HBM figure"
@@ -615,6 +618,9 @@ def other_workload_entry(hp, torch, dev, name, args, peak, rates=None):
     if args.parity:
         entry["parity"] = run.parity()
     run.release()
+    if args.probe:
+        rates = do_nothing_rates(hp, torch, dev, cfg)
+        entry["do_nothing"] = {**rates, **against_do_nothing(rates, share, entry["achieved"])}
     return entry
 
 
@@ -700,19 +706,19 @@ def run_gpu(args, cfg):
         parity = run.parity() if args.parity else None
         share = run.write_share(dominant)
         run.release()
-        rates = None
         if args.probe:
-            rates = do_nothing_rates(hp, torch, dev)
+            rates = do_nothing_rates(hp, torch, dev, cfg)
             roofline["do_nothing"] = {
-                "method": "hpsgd_probe_hbm: R read + W write arrays of 256 MB, one block per 128 groups of 8 floats, "
-                          "256-bit accesses, sums only; best of two runs of 10 timed launches each, CUDA events",
-                "rates": rates, **against_do_nothing(rates, share, kernels[dominant]["achieved"])}
+                "method": "hpsgd_probe_hbm: R read + W write arrays as long as one flat buffer of the workload (at most "
+                          "512 MB), one block per 128 groups of 8 floats, 256-bit accesses, sums only; best of two runs "
+                          "of `launches_timed` launches each, CUDA events",
+                **rates, **against_do_nothing(rates, share, kernels[dominant]["achieved"])}
         # ---- the other four workloads, briefly, each with its parity figures
         others = {}
         if args.other_workload_steps > 0 and not args.max_params:
             for name in workloads.names():
                 if name != cfg.name:
-                    others[name] = other_workload_entry(hp, torch, dev, name, args, peak, rates)
+                    others[name] = other_workload_entry(hp, torch, dev, name, args, peak)
         cpu = None
         if args.cpu_seconds > 0:
             eps, rounds, spent, desc, _ = oracle_sample_run(cfg, args.cpu_seconds)
