@@ -193,6 +193,47 @@ def oracle_sample_run(cfg, seconds, sample_params=4_000_000, min_rounds=2, max_r
     return cfg.K * P * rounds / spent, rounds, spent, desc, P
 
 
+def _oracle_range_worker(job):
+    """One process of oracle_all_cores: the oracle on parameters [lo, hi) of the workload, `rounds` rounds
+    timed after every process has its inputs (the barrier)."""
+    name, lo, hi, rounds, barrier = job
+    from oracle.ref import RefHPSGD
+    cfg = workloads.get(name)
+    idx = np.arange(lo, hi, dtype=np.int64)
+    o = RefHPSGD(idx.size, cfg.K, cfg.lr, cfg.momentum, cfg.weight_decay, cfg.staleness)
+    o.set_global(cfg.initial_global(idx))
+    grads = [[cfg.stored_gradient(i, t, idx) for i in range(cfg.K)] for t in range(2)]
+    barrier.wait()
+    t0 = time.perf_counter()
+    for r in range(rounds):
+        for i in range(cfg.K):
+            o.local_step(i, grads[r % 2][i])
+        o.sync_merge()
+    spent = time.perf_counter() - t0
+    o.close()
+    return spent
+
+
+def oracle_all_cores(cfg, per_core_params=1_000_000, rounds=12):
+    """The same oracle, unchanged, as one single-threaded process per host core, each on its own index
+    range of the workload (the path is independent per index, so the results are those of one process).
+    Processes are spawned, not forked: the parent has already used the GPU."""
+    import multiprocessing as mp
+    cores = os.cpu_count() or 1
+    per = min(per_core_params, cfg.P // cores)
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as manager:
+        barrier = manager.Barrier(cores)
+        jobs = [(cfg.name, j * per, (j + 1) * per, rounds, barrier) for j in range(cores)]
+        with ctx.Pool(cores) as pool:
+            times = pool.map(_oracle_range_worker, jobs, chunksize=1)
+    slowest = max(times)
+    return {"value": cfg.K * per * cores * rounds / slowest, "unit": UNIT, "cores": cores,
+            "sample": "%d processes x %d parameters each (the first %d of %s), all K=%d workers, %d rounds, "
+                      "slowest process" % (cores, per, per * cores, cfg.name, cfg.K, rounds),
+            "seconds": slowest}
+
+
 def run_reference(args, cfg):
     """--impl reference: the CPU oracle as it stands; each step is one round (K local steps + one
     merge) on a bounded sample of the workload, the first `--ref-sample` parameters."""
@@ -724,6 +765,8 @@ def run_gpu(args, cfg):
             eps, rounds, spent, desc, _ = oracle_sample_run(cfg, args.cpu_seconds)
             cpu = {"value": eps, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc,
                    "seconds": spent}
+            if args.cpu_all_cores and not args.max_params:
+                cpu["all_cores"] = oracle_all_cores(cfg)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": job_ms / args.steps, "higher_is_better": True,
@@ -822,6 +865,8 @@ def main():
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--e2e-host-buffers", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU oracle baseline budget (0 = skip)")
+    ap.add_argument("--cpu-all-cores", type=int, default=1,
+                    help="1: also time the oracle as one process per host core on disjoint index ranges")
     ap.add_argument("--other-workload-steps", type=int, default=10,
                     help="timed rounds for each of the other four workloads, reported under `workloads` (0 = skip)")
     ap.add_argument("--staging", type=int, default=0,

@@ -70,3 +70,15 @@ def test_roofline_byte_counts():
     assert bench.local_bytes_per_elem(workloads.get("cfg1")) == 12
     assert bench.local_bytes_per_elem(workloads.get("cfg4")) == 20
     assert bench.local_bytes_per_elem(workloads.get("cfg5")) == 18
+
+
+def test_oracle_on_all_cores_and_do_nothing_interpolation():
+    sys.path.insert(0, ROOT)
+    import bench
+    import workloads
+    out = bench.oracle_all_cores(workloads.get("cfg1"), per_core_params=20_000, rounds=2)
+    assert out["cores"] == os.cpu_count() and out["value"] > 0 and out["unit"] == "K*P elems/s"
+    rates = {"rates": [{"write_share": 0.0, "GB/s": 7500.0}, {"write_share": 0.5, "GB/s": 6800.0},
+                       {"write_share": 1.0, "GB/s": 7300.0}]}
+    got = bench.against_do_nothing(rates, 0.25, 3575.0)
+    assert got["do_nothing_GB/s"] == pytest.approx(7150.0) and got["kernel_over_do_nothing"] == pytest.approx(0.5)
