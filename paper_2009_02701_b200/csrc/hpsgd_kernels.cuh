@@ -803,7 +803,32 @@ __device__ __forceinline__ void round_rest(f8& acc, int& i, int K, const f8& wv,
     }
 }
 
+// One batch of `size` workers (1 <= size <= B), `size` the same for every thread of the launch: the
+// switch picks the instantiation whose register arrays have exactly that many entries.
 template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+__device__ __forceinline__ void round_batch_of(int size, f8& acc, bool first, const f8& wv, float* __restrict__ m,
+                                               int64_t stride, int i0, const BatchPtrs& gp, const SparseSeg& seg,
+                                               const SegPos& sp, int64_t o, const StepParams& p)
+{
+#define HPSGD_BATCH_CASE(S)                                                                                          \
+    case S:                                                                                                          \
+        if constexpr (S <= B) round_batch<S, BF16, MOM, WD, SPARSE, FROM_W>(acc, first, wv, m, stride, i0, gp, seg, sp, o, p, nullptr); \
+        break;
+    switch (size) {
+        HPSGD_BATCH_CASE(1) HPSGD_BATCH_CASE(2) HPSGD_BATCH_CASE(3) HPSGD_BATCH_CASE(4)
+        HPSGD_BATCH_CASE(5) HPSGD_BATCH_CASE(6) HPSGD_BATCH_CASE(7) HPSGD_BATCH_CASE(8)
+        HPSGD_BATCH_CASE(9) HPSGD_BATCH_CASE(10) HPSGD_BATCH_CASE(11) HPSGD_BATCH_CASE(12)
+        HPSGD_BATCH_CASE(13) HPSGD_BATCH_CASE(14) HPSGD_BATCH_CASE(15) HPSGD_BATCH_CASE(16)
+    default: break;
+    }
+#undef HPSGD_BATCH_CASE
+}
+
+// EVEN: K is not a multiple of B; the workers are then cut into ceil(K / B) batches of as equal a
+// size as possible (K = 11, B = 8: 6 + 5) instead of full batches and a tail (8 + 2 + 1), whose short
+// last batches leave a thread with almost nothing in flight (measured 5-15 % on K = 9, 11, 13, 15).
+// Launched only for such K; where B divides K the plain form below is used, unchanged.
+template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W, bool EVEN = false>
 __global__ void __launch_bounds__(kHotThreads, 2)
 round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m, int64_t stride, int K,
              BatchPtrs gp, SparseSeg seg, int64_t o0, int64_t n, int flags, StepParams p, int64_t lim)
@@ -817,7 +842,7 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         if (SPARSE) sp = seg_pos(seg, o);
         // the slot entries of the first two batches are requested before anything else: by the time
         // the gradient addresses are formed they have arrived (where the registers allow it)
-        constexpr bool PRE = SPARSE && FROM_W;
+        constexpr bool PRE = SPARSE && FROM_W && !EVEN;
         int32_t sl_pre[PRE ? 2 * B : 1];
         if (PRE && sp.inside && K >= B) {
 #pragma unroll
@@ -837,6 +862,15 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         // ---- local steps and the running sum of replica changes, worker 0 first
         f8 acc;
         int i = 0;
+        if constexpr (EVEN) {
+            const int batches = (K + B - 1) / B;
+            const int small = K / batches, larger = K - small * batches;      // `larger` batches hold small + 1 workers
+            for (int b = 0; b < batches; ++b) {
+                const int size = small + (b < larger ? 1 : 0);
+                round_batch_of<B, BF16, MOM, WD, SPARSE, FROM_W>(size, acc, i == 0, wv, m, stride, i, gp, seg, sp, o, p);
+                i += size;
+            }
+        } else {
         if (K >= B) {
             round_batch<B, BF16, MOM, WD, SPARSE, FROM_W>(acc, true, wv, m, stride, 0, gp, seg, sp, o, p, sl);
             i = B;
@@ -848,6 +882,7 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         for (; i + B <= K; i += B)
             round_batch<B, BF16, MOM, WD, SPARSE, FROM_W>(acc, false, wv, m, stride, i, gp, seg, sp, o, p, nullptr);
         round_rest<B / 2, BF16, MOM, WD, SPARSE, FROM_W>(acc, i, K, wv, m, stride, gp, seg, sp, o, p);
+        }
         // ---- merge
         f8 dnew, wn;
 #pragma unroll

@@ -251,8 +251,16 @@ int enqueue_merge(int flags)
             default: launch_accum_merge<0>(s, lo, hi - lo, flags); break;
             }
         } else if (lazy) {
+            // K up to 8 and K = 16 have instantiations of their own: with few workers the any-K form
+            // (built for many: two blocks per SM, eight loads at a time) keeps too little in flight
             switch (g.K) {
+            case 1: launch_merge_lazy<1>(s, rp, lo, hi - lo, flags); break;
+            case 2: launch_merge_lazy<2>(s, rp, lo, hi - lo, flags); break;
+            case 3: launch_merge_lazy<3>(s, rp, lo, hi - lo, flags); break;
             case 4: launch_merge_lazy<4>(s, rp, lo, hi - lo, flags); break;
+            case 5: launch_merge_lazy<5>(s, rp, lo, hi - lo, flags); break;
+            case 6: launch_merge_lazy<6>(s, rp, lo, hi - lo, flags); break;
+            case 7: launch_merge_lazy<7>(s, rp, lo, hi - lo, flags); break;
             case 8: launch_merge_lazy<8>(s, rp, lo, hi - lo, flags); break;
             case 16: launch_merge_lazy<16>(s, rp, lo, hi - lo, flags); break;
             default: launch_merge_lazy<0>(s, rp, lo, hi - lo, flags); break;
@@ -261,7 +269,13 @@ int enqueue_merge(int flags)
             TRY(launch_merge_staged(s, lo, hi - lo, flags));
         } else {
             switch (g.K) {
+            case 1: launch_merge<1>(s, lo, hi - lo, flags); break;
+            case 2: launch_merge<2>(s, lo, hi - lo, flags); break;
+            case 3: launch_merge<3>(s, lo, hi - lo, flags); break;
             case 4: launch_merge<4>(s, lo, hi - lo, flags); break;
+            case 5: launch_merge<5>(s, lo, hi - lo, flags); break;
+            case 6: launch_merge<6>(s, lo, hi - lo, flags); break;
+            case 7: launch_merge<7>(s, lo, hi - lo, flags); break;
             case 8: launch_merge<8>(s, lo, hi - lo, flags); break;
             case 16: launch_merge<16>(s, lo, hi - lo, flags); break;
             default: launch_merge<0>(s, lo, hi - lo, flags); break;
@@ -454,11 +468,40 @@ int enqueue_fused(const BatchPtrs& gp, bool sparse)
 }
 
 // ---------------------------------------------------------------------------- fuse 2: local step + merge, one round
+template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+void launch_round_b(const FusedLaunch& L)
+{
+    round_kernel<B, BF16, MOM, WD, SPARSE, FROM_W><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
+        g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
+}
+
+// The batch size is a template argument because it sizes the register arrays.  With fewer workers
+// than the largest batch holds, the instantiation for exactly K workers is used: all their loads are
+// in flight at once in a single batch, and the kernel needs only the registers of that batch, so
+// more blocks are resident per SM (with the largest batch, K = 1..7 reached 4.0-6.0 TB/s on large
+// models because a thread then has too little in flight for the few blocks its registers allow).
 template <bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 void launch_round(const FusedLaunch& L)
 {
     constexpr int B = round_batch_size(BF16, MOM, SPARSE, FROM_W);
-    round_kernel<B, BF16, MOM, WD, SPARSE, FROM_W><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
+    if constexpr (FROM_W) {
+        switch (g.K) {
+        case 1: return launch_round_b<1, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 2: return launch_round_b<2, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 3: return launch_round_b<3, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 4: return launch_round_b<4, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 5: return launch_round_b<5, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 6: return launch_round_b<6, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 7: return launch_round_b<7, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        default: break;
+        }
+    }
+    if (g.K % B == 0) return launch_round_b<B, BF16, MOM, WD, SPARSE, FROM_W>(L);
+    // B does not divide K: batches of as equal a size as possible instead of full batches and a tail
+    // (at most 8 workers per batch in this form: with 16 the bf16 + momentum variants spill, and the light
+    // variants, whose threads have little in flight anyway, gain more from the blocks that fewer registers allow)
+    constexpr int BE = B == 16 ? 8 : B;
+    round_kernel<BE, BF16, MOM, WD, SPARSE, FROM_W, true><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
         g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
 }
 

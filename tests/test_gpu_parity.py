@@ -487,6 +487,21 @@ def test_round_kernel_matches_oracle(K, momentum, wd, staleness, H):
                 session_kw=dict(lend_arena=True, canary=True, streams=True))
 
 
+@pytest.mark.parametrize("K", [1, 2, 3, 5, 6, 7, 9, 10, 11, 12, 13, 14, 15, 17, 20, 23, 24, 31])
+def test_round_kernel_any_worker_count(K):
+    """Every way the whole-round kernel cuts K workers into batches: fewer workers than a batch holds (one
+    batch of exactly K), a multiple of the batch size, and the rest (batches of as equal a size as possible),
+    for gradients and optimisers of different register weight, with one step per period (replicas read
+    from w) and with two (replica rows read)."""
+    for momentum, wd, dtype, H in ((0.9, 0.0, "f32", 1), (0.0, 0.0, "f32", 1), (0.9, 1e-3, "bf16", 1), (0.0, 0.0, "bf16", 1),
+                                   (0.9, 0.0, "f32", 2)):
+        cfg = small("round_k", K, [9001, 33, 1024], T=3, momentum=momentum, wd=wd, dtype=dtype)
+        gu.run_both(cfg, cfg.T, fuse=2, batched=True, steps_per_round=H)
+    for dtype in ("f32", "bf16"):
+        cfg = small("round_k_sparse", K, [520, 90 * 64, 77], T=3, dtype=dtype, sparse=(1, 90, 64), scale=1e-3)
+        gu.run_both(cfg, cfg.T, fuse=2, batched=True)
+
+
 @pytest.mark.parametrize("P", [1, 31, 33, 129, 1000, 4097])
 def test_round_kernel_odd_sizes(P):
     for K, momentum in ((2, 0.9), (7, 0.0), (16, 0.9)):
