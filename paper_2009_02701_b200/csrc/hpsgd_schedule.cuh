@@ -245,7 +245,13 @@ int enqueue_merge(int flags)
         TRY(prof_begin(s, (!lazy && staged_merge()) ? HPSGD_KERNEL_MERGE_STAGED : HPSGD_KERNEL_MERGE, &ep));
         if (g.form == HPSGD_FORM_GRADIENT_ACCUMULATION) {
             switch (g.K) {
+            case 1: launch_accum_merge<1>(s, lo, hi - lo, flags); break;
+            case 2: launch_accum_merge<2>(s, lo, hi - lo, flags); break;
+            case 3: launch_accum_merge<3>(s, lo, hi - lo, flags); break;
             case 4: launch_accum_merge<4>(s, lo, hi - lo, flags); break;
+            case 5: launch_accum_merge<5>(s, lo, hi - lo, flags); break;
+            case 6: launch_accum_merge<6>(s, lo, hi - lo, flags); break;
+            case 7: launch_accum_merge<7>(s, lo, hi - lo, flags); break;
             case 8: launch_accum_merge<8>(s, lo, hi - lo, flags); break;
             case 16: launch_accum_merge<16>(s, lo, hi - lo, flags); break;
             default: launch_accum_merge<0>(s, lo, hi - lo, flags); break;
@@ -325,7 +331,13 @@ int enqueue_pipelined_merge(int flags)
     EventPair ep2{};
     TRY(prof_begin(g.side, HPSGD_KERNEL_MERGE, &ep2));
     switch (g.K) {
+    case 1: launch_reduce<1>(g.wbuf[g.cur], rp, n); break;
+    case 2: launch_reduce<2>(g.wbuf[g.cur], rp, n); break;
+    case 3: launch_reduce<3>(g.wbuf[g.cur], rp, n); break;
     case 4: launch_reduce<4>(g.wbuf[g.cur], rp, n); break;
+    case 5: launch_reduce<5>(g.wbuf[g.cur], rp, n); break;
+    case 6: launch_reduce<6>(g.wbuf[g.cur], rp, n); break;
+    case 7: launch_reduce<7>(g.wbuf[g.cur], rp, n); break;
     case 8: launch_reduce<8>(g.wbuf[g.cur], rp, n); break;
     case 16: launch_reduce<16>(g.wbuf[g.cur], rp, n); break;
     default: launch_reduce<0>(g.wbuf[g.cur], rp, n); break;
