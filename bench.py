@@ -65,16 +65,16 @@ def fused_bytes_per_index(cfg):
 # the indices of that launch), keyed by (kernel, K, gradient dtype), with the SHA-1 of the kernel source the
 # capture was taken from.  A changed source voids them.
 NCU_TRAFFIC = {
-    # profiles/round_kernel_cfg4_cut16M.txt: 2.176083 GB read + 1.103313 GB written over 16,000,000 indices
-    ('round_kernel', 16, 'f32'): {"bytes_per_index": 3.279396e9 / 16e6, "source_sha1": "2fa64afb90ca87806f46c8a8e11ee16cbdb3c170"},
-    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200057 GB read + 2.123290 GB written over 16,000,000 indices
-    ('merge_step_kernel', 16, 'f32'): {"bytes_per_index": 5.323347e9 / 16e6, "source_sha1": "2fa64afb90ca87806f46c8a8e11ee16cbdb3c170"},
-    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152017 GB read + 1.093783 GB written over 16,000,000 indices
-    ('merge_kernel', 16, 'f32'): {"bytes_per_index": 2.245800e9 / 16e6, "source_sha1": "2fa64afb90ca87806f46c8a8e11ee16cbdb3c170"},
-    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072067 GB read + 1.992170 GB written over 16,000,000 indices
-    ('local_step_kernel', 16, 'f32'): {"bytes_per_index": 5.064237e9 / 16e6, "source_sha1": "2fa64afb90ca87806f46c8a8e11ee16cbdb3c170"},
-    # profiles/round_kernel_cfg3.txt: 1.843733 GB read + 0.974776 GB written over 25,600,000 indices
-    ('round_kernel', 8, 'f32'): {"bytes_per_index": 2.818509e9 / 25.6e6, "source_sha1": "2fa64afb90ca87806f46c8a8e11ee16cbdb3c170"},
+    # profiles/round_kernel_cfg4_cut16M.txt: 2.176072 GB read + 1.103841 GB written over 16,000,000 indices
+    ('round_kernel', 16, 'f32'): {"bytes_per_index": 3.279913e9 / 16e6, "source_sha1": "65baeb17746e2dd5628b51694946b71740efbca2"},
+    # profiles/merge_step_kernel_cfg4_cut16M.txt: 3.200026 GB read + 2.121919 GB written over 16,000,000 indices
+    ('merge_step_kernel', 16, 'f32'): {"bytes_per_index": 5.321945e9 / 16e6, "source_sha1": "65baeb17746e2dd5628b51694946b71740efbca2"},
+    # profiles/merge_kernel_cfg4_cut16M.txt: 1.152136 GB read + 1.094072 GB written over 16,000,000 indices
+    ('merge_kernel', 16, 'f32'): {"bytes_per_index": 2.246208e9 / 16e6, "source_sha1": "65baeb17746e2dd5628b51694946b71740efbca2"},
+    # profiles/local_step_kernel_cfg4_cut16M.txt: 3.072011 GB read + 1.991900 GB written over 16,000,000 indices
+    ('local_step_kernel', 16, 'f32'): {"bytes_per_index": 5.063911e9 / 16e6, "source_sha1": "65baeb17746e2dd5628b51694946b71740efbca2"},
+    # profiles/round_kernel_cfg3.txt: 1.843402 GB read + 0.974777 GB written over 25,600,000 indices
+    ('round_kernel', 8, 'f32'): {"bytes_per_index": 2.818179e9 / 25.6e6, "source_sha1": "65baeb17746e2dd5628b51694946b71740efbca2"},
 }
 
 

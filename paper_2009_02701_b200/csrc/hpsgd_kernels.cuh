@@ -775,14 +775,18 @@ __device__ __forceinline__ void round_batch(f8& acc, bool first, const f8& wv, f
 }
 
 // Workers whose loads are in flight together.  Each costs 8 registers for fp32 gradients (4 for
-// bf16), 8 for momentum and 8 for a replica row that has to be read; the batch is as large as
-// fits the 255 registers of a thread without spilling: 8 workers (16 x 32-byte loads) for the
-// usual fp32 + momentum case, 16 where a worker needs at most 12 registers.
+// bf16), 8 for momentum and 8 for a replica row that has to be read; without a sparse-row tensor the
+// batch is as large as fits the 255 registers of a thread without spilling: 8 workers (16 x 32-byte
+// loads) for the usual fp32 + momentum case, 16 where a worker needs at most 12 registers.  With a
+// sparse-row tensor small batches win: inside that tensor a gradient address waits for a row -> slot
+// entry, so what hides the latency is blocks per SM (fewer registers) and the next batch's requests,
+// not the width of one batch (batches of 4 against 8 on the GRU-shaped workload: K = 8 6.03 -> 6.81 TB/s,
+// K = 12 6.43 -> 6.83, K = 16 6.79 -> 6.83, K = 20 6.57 -> 6.82).
 constexpr int round_batch_size(bool bf16, bool mom, bool sparse, bool from_w)
 {
     const int per_worker = (bf16 ? 4 : 8) + (mom ? 8 : 0) + (from_w ? 0 : 8);
+    if (sparse) return 4;
     if (!from_w) return per_worker >= 24 ? 4 : 8;
-    if (sparse && (mom || !bf16)) return 8;          // the slot entries requested ahead take registers too
     return per_worker <= 12 ? 16 : 8;
 }
 
@@ -808,11 +812,11 @@ __device__ __forceinline__ void round_rest(f8& acc, int& i, int K, const f8& wv,
 template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 __device__ __forceinline__ void round_batch_of(int size, f8& acc, bool first, const f8& wv, float* __restrict__ m,
                                                int64_t stride, int i0, const BatchPtrs& gp, const SparseSeg& seg,
-                                               const SegPos& sp, int64_t o, const StepParams& p)
+                                               const SegPos& sp, int64_t o, const StepParams& p, const int32_t* pre)
 {
 #define HPSGD_BATCH_CASE(S)                                                                                          \
     case S:                                                                                                          \
-        if constexpr (S <= B) round_batch<S, BF16, MOM, WD, SPARSE, FROM_W>(acc, first, wv, m, stride, i0, gp, seg, sp, o, p, nullptr); \
+        if constexpr (S <= B) round_batch<S, BF16, MOM, WD, SPARSE, FROM_W>(acc, first, wv, m, stride, i0, gp, seg, sp, o, p, pre); \
         break;
     switch (size) {
         HPSGD_BATCH_CASE(1) HPSGD_BATCH_CASE(2) HPSGD_BATCH_CASE(3) HPSGD_BATCH_CASE(4)
@@ -842,7 +846,7 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
         if (SPARSE) sp = seg_pos(seg, o);
         // the slot entries of the first two batches are requested before anything else: by the time
         // the gradient addresses are formed they have arrived (where the registers allow it)
-        constexpr bool PRE = SPARSE && FROM_W && !EVEN;
+        constexpr bool PRE = SPARSE && FROM_W;
         int32_t sl_pre[PRE ? 2 * B : 1];
         if (PRE && sp.inside && K >= B) {
 #pragma unroll
@@ -867,7 +871,9 @@ round_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ m
             const int small = K / batches, larger = K - small * batches;      // `larger` batches hold small + 1 workers
             for (int b = 0; b < batches; ++b) {
                 const int size = small + (b < larger ? 1 : 0);
-                round_batch_of<B, BF16, MOM, WD, SPARSE, FROM_W>(size, acc, i == 0, wv, m, stride, i, gp, seg, sp, o, p);
+                // workers 0 .. 2B-1 had their slot entries requested above
+                round_batch_of<B, BF16, MOM, WD, SPARSE, FROM_W>(size, acc, i == 0, wv, m, stride, i, gp, seg, sp, o, p,
+                                                                 (PRE && i + size <= 2 * B) ? sl + i : nullptr);
                 i += size;
             }
         } else {

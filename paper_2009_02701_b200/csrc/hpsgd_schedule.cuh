@@ -487,34 +487,58 @@ void launch_round_b(const FusedLaunch& L)
         g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
 }
 
-// The batch size is a template argument because it sizes the register arrays.  With fewer workers
-// than the largest batch holds, the instantiation for exactly K workers is used: all their loads are
-// in flight at once in a single batch, and the kernel needs only the registers of that batch, so
-// more blocks are resident per SM (with the largest batch, K = 1..7 reached 4.0-6.0 TB/s on large
-// models because a thread then has too little in flight for the few blocks its registers allow).
+template <int B, bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
+void launch_round_even(const FusedLaunch& L)
+{
+    round_kernel<B, BF16, MOM, WD, SPARSE, FROM_W, true><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
+        g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
+}
+
+// The batch size is a template argument because it sizes the register arrays; which instantiation runs
+// depends on K.
+//   Without a sparse-row tensor: fewer workers than the largest batch holds use the instantiation for
+//   exactly K workers - all their loads in flight at once in a single batch, and only the registers of
+//   that batch, so more blocks are resident per SM (with the largest batch, K = 1..7 reached 4.0-6.0 TB/s
+//   on large models: too little in flight per thread for the few blocks its registers allow).  Where the
+//   largest batch divides K, full batches; otherwise batches of as equal a size as possible.
+//   With a sparse-row tensor: at least two batches of at most four workers (round_batch_size says why).
 template <bool BF16, bool MOM, bool WD, bool SPARSE, bool FROM_W>
 void launch_round(const FusedLaunch& L)
 {
     constexpr int B = round_batch_size(BF16, MOM, SPARSE, FROM_W);
-    if constexpr (FROM_W) {
-        switch (g.K) {
+    const int K = g.K;
+    if constexpr (SPARSE) {
+        static_assert(B == 4, "the cases below are written for batches of four");
+        if (K >= 7) return K % 4 == 0 ? launch_round_b<4, BF16, MOM, WD, SPARSE, FROM_W>(L)
+                                      : launch_round_even<4, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        switch (K) {                                   // two batches: ceil(K / 2) and the rest
         case 1: return launch_round_b<1, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 2: return launch_round_b<2, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 3: return launch_round_b<3, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 4: return launch_round_b<4, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 5: return launch_round_b<5, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 6: return launch_round_b<6, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        case 7: return launch_round_b<7, BF16, MOM, WD, SPARSE, FROM_W>(L);
-        default: break;
+        case 2: return launch_round_b<1, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 3: return launch_round_even<2, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 4: return launch_round_b<2, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        case 5: return launch_round_even<3, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        default: return launch_round_b<3, BF16, MOM, WD, SPARSE, FROM_W>(L);      // 6
         }
+    } else {
+        if constexpr (FROM_W) {
+            switch (K) {
+            case 1: return launch_round_b<1, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 2: return launch_round_b<2, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 3: return launch_round_b<3, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 4: return launch_round_b<4, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 5: return launch_round_b<5, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 6: return launch_round_b<6, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            case 7: return launch_round_b<7, BF16, MOM, WD, SPARSE, FROM_W>(L);
+            default: break;
+            }
+        }
+        if (K % B == 0) return launch_round_b<B, BF16, MOM, WD, SPARSE, FROM_W>(L);
+        // at most 8 workers per batch in the evenly split form: with 16 the bf16 + momentum variants spill,
+        // and the light variants, whose threads have little in flight anyway, gain more from the blocks
+        // that fewer registers allow
+        constexpr int BE = B == 16 ? 8 : B;
+        launch_round_even<BE, BF16, MOM, WD, SPARSE, FROM_W>(L);
     }
-    if (g.K % B == 0) return launch_round_b<B, BF16, MOM, WD, SPARSE, FROM_W>(L);
-    // B does not divide K: batches of as equal a size as possible instead of full batches and a tail
-    // (at most 8 workers per batch in this form: with 16 the bf16 + momentum variants spill, and the light
-    // variants, whose threads have little in flight anyway, gain more from the blocks that fewer registers allow)
-    constexpr int BE = B == 16 ? 8 : B;
-    round_kernel<BE, BF16, MOM, WD, SPARSE, FROM_W, true><<<hot_grid(L.n), kHotThreads, 0, g.main>>>(
-        g.w, g.D, g.m, g.stride, g.K, L.gp, L.seg, L.o0, L.n, L.flags, L.p, group_limit());
 }
 
 template <bool BF16, bool MOM, bool WD>
