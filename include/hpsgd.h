@@ -94,9 +94,14 @@ enum {
                                    memory traffic can be timed against each other on the same state; the merge has
                                    no data reuse for shared memory to exploit, and the plain form is as fast or
                                    faster.  The staged kernel is the only device code of this library that waits
-                                   (on its own loads, a bounded number of tries): if a wait ever runs out, the
+                                   (on its own loads, for one second at most): if a wait ever runs out, the
                                    block writes nothing and the next call that waits for the device returns
                                    HPSGD_E_TIMEOUT. */
+    HPSGD_OPT_DEBUG_STAGE_STALL = 10, /* Checked build only; HPSGD_E_UNSUPPORTED otherwise.  1: the barrier of the staged
+                                   merge (HPSGD_OPT_STAGING) is told to expect 16 bytes more than its copies bring,
+                                   so that its wait runs out after one second: the way to see the time-out path
+                                   (blocks write nothing, the next synchronisation returns HPSGD_E_TIMEOUT) without
+                                   a fault.  The state is not consistent afterwards; destroy it. */
     HPSGD_OPT_DEBUG_GROUP_LIMIT = 8 /* Checked build (compiled with -DHPSGD_DEBUG) only; HPSGD_E_UNSUPPORTED
                                    otherwise.  In that build every hot kernel tests each 8-element group
                                    index against the number of groups of a flat buffer before touching

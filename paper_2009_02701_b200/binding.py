@@ -18,6 +18,7 @@ HPSGD_OPT_WEIGHT_DECAY, HPSGD_OPT_STALENESS, HPSGD_OPT_GRAD_DTYPE = 1, 2, 3
 HPSGD_OPT_OVERLAP, HPSGD_OPT_CHUNKS, HPSGD_OPT_PROFILE, HPSGD_OPT_FUSE = 4, 5, 6, 7
 HPSGD_OPT_DEBUG_GROUP_LIMIT = 8
 HPSGD_OPT_STAGING = 9
+HPSGD_OPT_DEBUG_STAGE_STALL = 10
 HPSGD_KERNEL_LOCAL_STEP, HPSGD_KERNEL_MERGE, HPSGD_KERNEL_MERGE_STEP, HPSGD_KERNEL_ROUND = 0, 1, 2, 3
 HPSGD_KERNEL_MERGE_STAGED = 4
 HPSGD_F32, HPSGD_BF16 = 0, 1

@@ -272,6 +272,14 @@ int hpsgd_set_option(int key, double value)
 #else
         return fail(HPSGD_E_UNSUPPORTED, "only the checked build (HPSGD_DEBUG) has kernel guards");
 #endif
+    case HPSGD_OPT_DEBUG_STAGE_STALL:
+#ifdef HPSGD_DEBUG
+        if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "stall must be 0 or 1");
+        g.debug_stage_stall = value != 0.0;
+        return HPSGD_OK;
+#else
+        return fail(HPSGD_E_UNSUPPORTED, "only the checked build (HPSGD_DEBUG) can make the staged merge's wait run out");
+#endif
     case HPSGD_OPT_PROFILE:
         if (value != 0.0 && value != 1.0) return fail(HPSGD_E_BADARG, "profile must be 0 or 1");
         TRY(prof_resolve());

@@ -201,7 +201,8 @@ int launch_merge_staged(cudaStream_t s, int64_t o0, int64_t n, int flags)
         g.staged_attr = true;
     }
     const int64_t tiles = (n + kStageGroups - 1) / kStageGroups;
-    merge_staged_kernel<<<(unsigned)tiles, kHotThreads, smem, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags, group_limit());
+    merge_staged_kernel<<<(unsigned)tiles, kHotThreads, smem, s>>>(g.w, g.D, g.r, g.stride, g.K, o0, n, flags, group_limit(),
+                                                                   g.debug_stage_stall ? 16u : 0u);
     g.staged_ran = true;
     return HPSGD_OK;
 }

@@ -13,8 +13,8 @@
 //                         with that share of writes (hpsgd_probe_hbm).
 //
 // The staged kernel is the one place in the library where device code waits: on the mbarrier
-// its own bulk loads complete on.  The wait is a bounded try_wait loop; a block whose wait runs
-// out counts itself in g_stage_timeouts, waits once more (bounded) so that no copy is still on
+// its own bulk loads complete on.  The wait is a try_wait loop bounded by time (one second); a block
+// whose wait runs out counts itself in g_stage_timeouts, waits once more (bounded) so that no copy is still on
 // its way into shared memory that the next block will own, writes nothing and returns.  The
 // host turns a non-zero count into HPSGD_E_TIMEOUT at its next synchronisation.  Blocks are
 // launched without clusters and every copy is between this GPU's global memory and the issuing
@@ -27,7 +27,7 @@ namespace hpsgd {
 
 constexpr int kStageGroups = 128;               // 8-element groups per tile: 4 KB per array
 constexpr int kStageTileFloats = kStageGroups * 8;
-constexpr uint32_t kStageWaitTries = 1u << 22;  // try_wait calls (each blocks for a hardware-chosen slice of time)
+constexpr uint64_t kStageWaitNs = 1000000000ull;   // how long a block waits for its own loads: one second
 
 __device__ unsigned int g_stage_timeouts;       // blocks whose wait for their own loads ran out
 
@@ -50,19 +50,28 @@ __device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src,
                  : "memory");
 }
 
-// Bounded wait for phase `parity` of the barrier: true when the phase completed.
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait for phase `parity` of the barrier: true when the phase completed, false when
+// kStageWaitNs went by first (each try_wait itself returns after a hardware-chosen slice of time).
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity)
 {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t tries = 0; tries < kStageWaitTries; ++tries) {
+    const uint64_t t0 = global_ns();
+    for (;;) {
         uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
+        if (global_ns() - t0 > kStageWaitNs) return false;
     }
-    return false;
 }
 
 // One block per tile of kStageGroups groups.  Shared memory: [(K + 2)][kStageTileFloats] floats,
@@ -71,7 +80,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity)
 // the operations per element and their order are those of merge_kernel.
 __global__ void __launch_bounds__(kHotThreads)
 merge_staged_kernel(float* __restrict__ w, float* __restrict__ D, float* __restrict__ r, int64_t stride,
-                    int K, int64_t o0, int64_t n, int flags, int64_t lim)
+                    int K, int64_t o0, int64_t n, int flags, int64_t lim, uint32_t never_arriving_bytes)
 {
     extern __shared__ __align__(128) float tiles[];
     __shared__ __align__(8) uint64_t bar;
@@ -94,7 +103,9 @@ merge_staged_kernel(float* __restrict__ w, float* __restrict__ D, float* __restr
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        const uint32_t expect = bytes * (uint32_t)(K + 1 + (pending ? 1 : 0));
+        // never_arriving_bytes is 0 except in the checked build's test of the time-out path, where the
+        // barrier is told to expect bytes that no copy brings, so that the wait below runs out
+        const uint32_t expect = bytes * (uint32_t)(K + 1 + (pending ? 1 : 0)) + never_arriving_bytes;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(&bar)), "r"(expect) : "memory");
         bulk_load(tiles, w + e0, bytes, &bar);
         if (pending) bulk_load(tiles + kStageTileFloats, D + e0, bytes, &bar);

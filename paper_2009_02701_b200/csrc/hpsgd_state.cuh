@@ -130,6 +130,7 @@ struct Ctx {
     std::vector<EventPair> prof;           // profiling
     double prof_ms[5] = {0, 0, 0, 0, 0};
     int64_t prof_launches[5] = {0, 0, 0, 0, 0};
+    bool debug_stage_stall = false;        // checked build: the staged merge's barrier expects bytes that never arrive
     int64_t debug_limit = -1;              // checked build: groups per flat buffer the kernels test against (< 0: P_pad / 8)
 } g;
 
@@ -172,7 +173,7 @@ int staged_poll()
     if (n != 0) {
         const unsigned int zero = 0;
         CUDA_TRY(cudaMemcpyToSymbol(g_stage_timeouts, &zero, sizeof zero));
-        return fail(HPSGD_E_TIMEOUT, "staged merge: %u blocks gave up waiting for their bulk loads and wrote nothing; "
+        return fail(HPSGD_E_TIMEOUT, "staged merge: %u blocks gave up waiting for their bulk loads after one second and wrote nothing; "
                                      "the state is no longer consistent", n);
     }
     return HPSGD_OK;

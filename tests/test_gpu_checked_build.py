@@ -136,9 +136,44 @@ def test_kernel_guard_records_and_skips(checked_library, fuse, batched, staging)
         assert bool(torch.isfinite(gu.dev_view(hp.hpsgd_get_global(), cfg.layout.P_pad)).all())
 
 
+def test_staged_merge_wait_that_runs_out_is_reported(checked_library):
+    """The one device-side wait of the library (the staged merge waiting for its own bulk loads) is bounded:
+    with its barrier told to expect bytes that never arrive, every block gives up after a second, writes
+    nothing, and the next synchronisation returns HPSGD_E_TIMEOUT; the context stays usable."""
+    import time
+    cfg = small("chk_stall", 3, [2000, 40], T=1)           # three tiles, three blocks
+    with gu.session(cfg, staging=1):
+        keep = []
+        for i in range(cfg.K):
+            gu.gpu_step(cfg, i, gu.host_inputs(cfg, i, 0), keep)
+        hp.hpsgd_synchronize()
+        n = cfg.layout.P_pad
+        w_before = gu.dev_view(hp.hpsgd_get_global(), n)
+        rows = [hp.hpsgd_get_replica(i)[0] for i in range(cfg.K)]
+        r_before = [gu.dev_view(r, n) for r in rows]
+        hp.hpsgd_set_option(hp.HPSGD_OPT_DEBUG_STAGE_STALL, 1)
+        hp.hpsgd_sync_merge()
+        t0 = time.perf_counter()
+        with pytest.raises(hp.HpsgdError) as err:
+            hp.hpsgd_synchronize()
+        waited = time.perf_counter() - t0
+        assert err.value.code == hp.HPSGD_E_TIMEOUT and "gave up waiting" in hp.last_error()
+        assert 1.0 < waited < 30.0
+        hp.hpsgd_set_option(hp.HPSGD_OPT_DEBUG_STAGE_STALL, 0)
+        hp.hpsgd_synchronize()                               # reported once
+        assert torch.equal(gu.dev_view(hp.hpsgd_get_global(), n), w_before), "a block that gave up wrote w"
+        for r, before in zip(rows, r_before):
+            assert torch.equal(gu.dev_view(r, n), before), "a block that gave up wrote a replica"
+    # and the library carries on: the same kernel, unstalled, against the oracle
+    gu.run_both(small("chk_after_stall", 3, [2000, 40], T=2), 2, session_kw=dict(staging=1))
+
+
 def test_normal_build_has_no_guard_option():
     cfg = small("chk_none", 2, [1000])
     with gu.session(cfg):
         with pytest.raises(hp.HpsgdError) as err:
             hp.hpsgd_set_option(hp.HPSGD_OPT_DEBUG_GROUP_LIMIT, 10)
+        assert err.value.code == hp.HPSGD_E_UNSUPPORTED
+        with pytest.raises(hp.HpsgdError) as err:
+            hp.hpsgd_set_option(hp.HPSGD_OPT_DEBUG_STAGE_STALL, 1)
         assert err.value.code == hp.HPSGD_E_UNSUPPORTED
